@@ -1,0 +1,166 @@
+/*
+ * refreekv.h - C ABI of the B200 (sm_100a) post-prefill KV-cache compression
+ * pass of ReFreeKV (arXiv 2502.16886).
+ *
+ * For every (sequence s, KV head g) of one Transformer layer the pass
+ *   (a) scores each cached position by the softmax attention it receives from
+ *       the last `window` queries of the prompt (the reduced attention vector
+ *       A' of Section 3.2, Eq. 2, averaged over the query heads of the KV head),
+ *   (b) ranks the positions (Section 3.2 "Initial Ranking", or by score as in
+ *       Section 4.4) and applies the threshold-free stopping rule (Eq. 1, in
+ *       its cumulative form Eq. 3) to choose a budget b,
+ *   (c) copies the kept K and V rows, in their original order, into a dense
+ *       ragged cache (the "Compress" steps of Algorithm 1).
+ *
+ * Conventions common to every entry point
+ *   - All array arguments are DEVICE pointers owned by the caller unless the
+ *     function name ends in `_host`.  The library allocates nothing, never
+ *     synchronises the device (except the `_host` variant), and enqueues all
+ *     work on the caller's stream (`stream` is a cudaStream_t passed as void*).
+ *   - Element (s, g, i, :) of K lives at
+ *       k + s*k_stride_seq + (seq_start[s] + i)*k_stride_tok + g*k_stride_head
+ *     (strides in elements, head_dim contiguous); V likewise.  Rows
+ *     [0, kv_tokens) of the token axis must be readable for every (s, g).
+ *   - q_win is [num_seqs, num_q_heads, window, head_dim] contiguous;
+ *     q_win[s, h, r, :] is the query at position seq_len[s] - window + r; rows
+ *     with a negative position are ignored.
+ *   - Per-position arrays (scores) are [num_kv_heads, total_tokens], sequences
+ *     packed along the token axis by the running sum of seq_len;
+ *     total_tokens = sum of seq_len.
+ *   - Unit u = s*num_kv_heads + g owns rows [offsets[u], offsets[u+1]) of
+ *     k_out / v_out / kept_idx; lengths[u] = offsets[u+1] - offsets[u].
+ *   - The return value reports errors the host can see (bad arguments,
+ *     unsupported shapes, workspace too small, CUDA launch failures); nothing
+ *     is launched when it is not REFREE_OK.  Conditions only the device can
+ *     see are OR-ed into *device_status (nullable, int32, caller zeroes it):
+ *       REFREE_DEV_CAPACITY  output rows would exceed capacity_rows (nothing is
+ *                            written past capacity)
+ *       REFREE_DEV_TIMEOUT   a bounded on-device wait gave up
+ *       REFREE_DEV_NONFINITE a score was NaN or infinite
+ */
+#ifndef REFREEKV_H
+#define REFREEKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    REFREE_OK = 0,
+    REFREE_ERR_INVALID_ARG = 1,
+    REFREE_ERR_UNSUPPORTED = 2,
+    REFREE_ERR_WORKSPACE = 3,
+    REFREE_ERR_CAPACITY = 4,
+    REFREE_ERR_CUDA = 5,
+    REFREE_ERR_TIMEOUT = 6,
+    REFREE_ERR_NONFINITE = 7
+} refree_status;
+
+enum { REFREE_DEV_CAPACITY = 1, REFREE_DEV_TIMEOUT = 2, REFREE_DEV_NONFINITE = 4 };
+
+enum { REFREE_RANK_POSITION = 0, REFREE_RANK_SCORE = 1 };
+enum { REFREE_SCOPE_HEAD = 0, REFREE_SCOPE_LAYER = 1 };
+enum { REFREE_DTYPE_F32 = 0, REFREE_DTYPE_BF16 = 1 };
+
+typedef struct {
+    int32_t num_seqs, num_q_heads, num_kv_heads, head_dim; /* Hq % Hkv == 0; head_dim 64 or 128 */
+    int32_t window;      /* w >= 1: trailing query rows, the paper's k (default 1, Section 4.1)   */
+    int32_t sink;        /* m >= 0: leading positions ranked first (default 4, Section 4.1)       */
+    float   threshold;   /* T in [0, 1): universal threshold of Eq. 1 (default 0.01, Section 3.2) */
+    int32_t rank_mode;   /* REFREE_RANK_POSITION (Section 3.2) or REFREE_RANK_SCORE (Section 4.4) */
+    int32_t scope;       /* one budget per (sequence, KV head), or one per sequence for the layer */
+    int32_t keep_window; /* 1: budget never below min(n, m + min(w, n))                          */
+    int32_t force_full;  /* 1: keep everything (the frozen bottom layers of Section 3.3)          */
+    int32_t dtype;       /* REFREE_DTYPE_*: type of q_win, K, V and of k_out, v_out               */
+    int64_t kv_tokens;   /* readable extent of the token axis of K and V                          */
+    int64_t k_stride_seq, k_stride_tok, k_stride_head;
+    int64_t v_stride_seq, v_stride_tok, v_stride_head;
+} refree_params;
+
+/* Defaults of the paper (Section 3.2, Section 4.1): w = 1, m = 4, T = 1 %,
+ * position ranking, per-head budgets, window floor on, bf16.  Shapes and
+ * strides are left zero for the caller to fill. */
+void refree_default_params(refree_params *p);
+
+/* Bytes of device scratch that score / select / compress_layer need for this
+ * shape.  `bytes` (host pointer) receives the size; pass a buffer at least
+ * that large, 256-byte aligned, as `workspace`.  Contents need no
+ * initialisation and are not preserved between calls. */
+refree_status refree_workspace_size(const refree_params *p, int64_t total_tokens, size_t *bytes);
+
+/* Steps S1-S3: reduced attention A' (Eq. 2) of every position, for every KV
+ * head, from the causal softmax of the window queries (Algorithm 1,
+ * "Attention" step; Section 3.2 "Reducing Overhead").
+ *   scores [num_kv_heads, total_tokens] fp32, written in full. */
+refree_status refree_score(const refree_params *p, const void *q_win, const void *k,
+                           const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                           float *scores, void *workspace, size_t workspace_bytes,
+                           int32_t *device_status, void *stream);
+
+/* Steps S4-S6: rank the positions, evaluate the stopping rule (Eq. 1 / Eq. 3;
+ * Algorithm 1 Square .. Where) in fp64 over the squares of the fp32 scores,
+ * apply the window floor, and emit the kept set in ascending position order.
+ *   lengths  [num_seqs * num_kv_heads] int32
+ *   offsets  [num_seqs * num_kv_heads + 1] int64, running sum of lengths
+ *   kept_idx [capacity_rows] int32 positions within their sequence (nullable:
+ *            then only lengths and offsets are produced) */
+refree_status refree_select_budget(const refree_params *p, const float *scores,
+                                   const int32_t *seq_len, int64_t total_tokens,
+                                   int32_t *lengths, int64_t *offsets,
+                                   int32_t *kept_idx, int64_t capacity_rows,
+                                   void *workspace, size_t workspace_bytes,
+                                   int32_t *device_status, void *stream);
+
+/* Step S7: K_c[offsets[u] + t, :] = K[s, kept_idx[offsets[u] + t], g, :], the
+ * same for V; rows are copied bit for bit (Algorithm 1 "Compress" steps).
+ *   k_out, v_out [capacity_rows, head_dim], must not overlap K or V. */
+refree_status refree_compact(const refree_params *p, const void *k, const void *v,
+                             const int32_t *seq_start, const int32_t *seq_len,
+                             const int32_t *lengths, const int64_t *offsets,
+                             const int32_t *kept_idx, void *k_out, void *v_out,
+                             int64_t capacity_rows, int32_t *device_status, void *stream);
+
+/* The whole per-layer pass of Algorithm 1 (everything after the prefill of the
+ * layer): score -> select -> compact, enqueued back to back with no host
+ * synchronisation.  kept_idx and scores are nullable (scratch is used then).
+ * Worst-case capacity_rows is num_kv_heads * total_tokens. */
+refree_status refree_compress_layer(const refree_params *p, const void *q_win,
+                                    const void *k, const void *v,
+                                    const int32_t *seq_start, const int32_t *seq_len,
+                                    int64_t total_tokens,
+                                    void *k_out, void *v_out, int64_t capacity_rows,
+                                    int32_t *lengths, int64_t *offsets,
+                                    int32_t *kept_idx, float *scores,
+                                    void *workspace, size_t workspace_bytes,
+                                    int32_t *device_status, void *stream);
+
+/* The same pass of Algorithm 1 for callers whose cache lives in HOST memory
+ * (pinned or pageable): q_win, k, v, seq_start, seq_len are host pointers, and
+ * so are the outputs k_out, v_out (capacity_rows rows), lengths, offsets,
+ * kept_idx (nullable) and scores (nullable).  k and v are read over `kv_elems`
+ * elements each (the size of the caller's arrays).  `arena` is a DEVICE buffer
+ * of at least refree_host_arena_size() bytes that stages inputs, outputs and
+ * scratch; the call copies in, runs the pass, copies the kept rows back and
+ * synchronises `stream` before returning.  Device-side conditions are
+ * returned as REFREE_ERR_CAPACITY / _TIMEOUT / _NONFINITE. */
+refree_status refree_host_arena_size(const refree_params *p, int64_t total_tokens,
+                                     int64_t kv_elems, int64_t capacity_rows, size_t *bytes);
+refree_status refree_compress_layer_host(const refree_params *p, const void *q_win,
+                                         const void *k, const void *v, int64_t kv_elems,
+                                         const int32_t *seq_start, const int32_t *seq_len,
+                                         int64_t total_tokens,
+                                         void *k_out, void *v_out, int64_t capacity_rows,
+                                         int32_t *lengths, int64_t *offsets,
+                                         int32_t *kept_idx, float *scores,
+                                         void *arena, size_t arena_bytes, void *stream);
+
+/* Static string for a status code. */
+const char *refree_status_string(refree_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REFREEKV_H */

@@ -1,0 +1,251 @@
+"""ctypes binding of ``librefreekv.so``: same names as the C ABI, argument
+marshalling only.  Every step of the pass runs in the CUDA kernels of the
+library; there is no CPU fallback, and a missing library is an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+from typing import Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "librefreekv.so")
+
+REFREE_OK = 0
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CAPACITY", "CUDA", "TIMEOUT", "NONFINITE"]
+DEV_CAPACITY, DEV_TIMEOUT, DEV_NONFINITE = 1, 2, 4
+RANK_POSITION, RANK_SCORE = 0, 1
+SCOPE_HEAD, SCOPE_LAYER = 0, 1
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+
+class RefreeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        name = STATUS_NAMES[code] if 0 <= code < len(STATUS_NAMES) else str(code)
+        super().__init__(f"{where}: REFREE_ERR_{name} ({status_string(code)})")
+
+
+class CParams(ctypes.Structure):
+    _fields_ = [
+        ("num_seqs", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("window", ctypes.c_int32), ("sink", ctypes.c_int32),
+        ("threshold", ctypes.c_float),
+        ("rank_mode", ctypes.c_int32), ("scope", ctypes.c_int32),
+        ("keep_window", ctypes.c_int32), ("force_full", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("kv_tokens", ctypes.c_int64),
+        ("k_stride_seq", ctypes.c_int64), ("k_stride_tok", ctypes.c_int64), ("k_stride_head", ctypes.c_int64),
+        ("v_stride_seq", ctypes.c_int64), ("v_stride_tok", ctypes.c_int64), ("v_stride_head", ctypes.c_int64),
+    ]
+
+
+@dataclasses.dataclass
+class Params:
+    """Mirror of ``refree_params`` (see ``include/refreekv.h``)."""
+    num_seqs: int
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int
+    window: int = 1
+    sink: int = 4
+    threshold: float = 0.01
+    rank_mode: int = RANK_POSITION
+    scope: int = SCOPE_HEAD
+    keep_window: int = 1
+    force_full: int = 0
+    dtype: int = DTYPE_BF16
+    kv_tokens: int = 0
+    k_strides: tuple = (0, 0, 0)   # (seq, tok, head) in elements
+    v_strides: tuple = (0, 0, 0)
+
+    def c_struct(self) -> CParams:
+        return CParams(self.num_seqs, self.num_q_heads, self.num_kv_heads, self.head_dim,
+                       self.window, self.sink, self.threshold, self.rank_mode, self.scope,
+                       self.keep_window, self.force_full, self.dtype, self.kv_tokens,
+                       *self.k_strides, *self.v_strides)
+
+
+_LIB = None
+_VP, _I64, _SZ = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+_PP = ctypes.POINTER(CParams)
+
+SIGNATURES = {
+    "refree_default_params": (None, [_PP]),
+    "refree_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "refree_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
+    "refree_score": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
+    "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
+    "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
+                                             _VP, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_host_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
+    "refree_compress_layer_host": (ctypes.c_int, [_PP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP, _I64,
+                                                  _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+}
+
+
+def lib():
+    """Load the CUDA library (once).  Raises if it has not been built."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2502_16886_b200.build` "
+                "(there is no CPU fallback)")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _LIB = handle
+    return _LIB
+
+
+def status_string(code: int) -> str:
+    return lib().refree_status_string(int(code)).decode()
+
+
+def default_params() -> CParams:
+    c = CParams()
+    lib().refree_default_params(ctypes.byref(c))
+    return c
+
+
+def _dp(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != REFREE_OK:
+        raise RefreeError(code, where)
+
+
+def refree_workspace_size(p: Params, total_tokens: int) -> int:
+    out = _SZ(0)
+    c = p.c_struct()
+    _check(lib().refree_workspace_size(ctypes.byref(c), total_tokens, ctypes.byref(out)), "refree_workspace_size")
+    return int(out.value)
+
+
+def refree_score(p: Params, q_win, k, seq_start, seq_len, total_tokens, scores, workspace,
+                 device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_score(ctypes.byref(c), _dp(q_win), _dp(k), _dp(seq_start), _dp(seq_len), total_tokens,
+                            _dp(scores), _dp(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                            _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_score")
+    return rc
+
+
+def refree_select_budget(p: Params, scores, seq_len, total_tokens, lengths, offsets, kept_idx, capacity_rows,
+                         workspace, device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_select_budget(ctypes.byref(c), _dp(scores), _dp(seq_len), total_tokens, _dp(lengths),
+                                    _dp(offsets), _dp(kept_idx), capacity_rows, _dp(workspace),
+                                    workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                    _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_select_budget")
+    return rc
+
+
+def refree_compact(p: Params, k, v, seq_start, seq_len, lengths, offsets, kept_idx, k_out, v_out, capacity_rows,
+                   device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_compact(ctypes.byref(c), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len), _dp(lengths),
+                              _dp(offsets), _dp(kept_idx), _dp(k_out), _dp(v_out), capacity_rows,
+                              _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compact")
+    return rc
+
+
+def refree_compress_layer(p: Params, q_win, k, v, seq_start, seq_len, total_tokens, k_out, v_out, capacity_rows,
+                          lengths, offsets, kept_idx, scores, workspace, device_status=None, stream=None,
+                          check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_compress_layer(ctypes.byref(c), _dp(q_win), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len),
+                                     total_tokens, _dp(k_out), _dp(v_out), capacity_rows, _dp(lengths),
+                                     _dp(offsets), _dp(kept_idx), _dp(scores), _dp(workspace),
+                                     workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                     _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compress_layer")
+    return rc
+
+
+def refree_host_arena_size(p: Params, total_tokens: int, kv_elems: int, capacity_rows: int) -> int:
+    out = _SZ(0)
+    c = p.c_struct()
+    _check(lib().refree_host_arena_size(ctypes.byref(c), total_tokens, kv_elems, capacity_rows, ctypes.byref(out)),
+           "refree_host_arena_size")
+    return int(out.value)
+
+
+def refree_compress_layer_host(p: Params, q_win, k, v, seq_start, seq_len, total_tokens, k_out, v_out,
+                               capacity_rows, lengths, offsets, kept_idx, scores, arena, stream=None,
+                               check=True) -> int:
+    """All tensors but ``arena`` are CPU tensors (pinned or pageable)."""
+    c = p.c_struct()
+    rc = lib().refree_compress_layer_host(ctypes.byref(c), _dp(q_win), _dp(k), _dp(v), k.numel(), _dp(seq_start),
+                                          _dp(seq_len), total_tokens, _dp(k_out), _dp(v_out), capacity_rows,
+                                          _dp(lengths), _dp(offsets), _dp(kept_idx), _dp(scores), _dp(arena),
+                                          arena.numel() * arena.element_size(), _stream(stream))
+    if check:
+        _check(rc, "refree_compress_layer_host")
+    return rc
+
+
+# ---- convenience wrapper -----------------------------------------------------
+@dataclasses.dataclass
+class LayerResult:
+    k_out: torch.Tensor
+    v_out: torch.Tensor
+    lengths: torch.Tensor     # int32 [B, Hkv]
+    offsets: torch.Tensor     # int64 [B*Hkv + 1]
+    kept_idx: Optional[torch.Tensor]
+    scores: Optional[torch.Tensor]
+    device_status: torch.Tensor
+
+
+def params_for(cfg, layer_cache, **overrides) -> Params:
+    """``Params`` for a ``workloads.LayerCache`` (strides in elements)."""
+    ss, st, sh = layer_cache.strides()
+    p = Params(num_seqs=int(layer_cache.seq_len.numel()), num_q_heads=cfg.num_q_heads,
+               num_kv_heads=cfg.num_kv_heads, head_dim=cfg.head_dim, window=cfg.window, sink=cfg.sink,
+               dtype=DTYPE_F32 if cfg.dtype == "fp32" else DTYPE_BF16,
+               kv_tokens=layer_cache.total_tokens, k_strides=(ss, st, sh), v_strides=(ss, st, sh))
+    for key, val in overrides.items():
+        setattr(p, key, val)
+    return p
+
+
+def compress_layer(p: Params, q_win, k, v, seq_start, seq_len, total_tokens, want_scores=True,
+                   want_kept_idx=True, capacity_rows=None, workspace=None, stream=None) -> LayerResult:
+    """Allocate outputs with torch and run the fused pass on device tensors."""
+    dev = k.device
+    cap = p.num_kv_heads * total_tokens if capacity_rows is None else capacity_rows
+    k_out = torch.empty(max(cap, 1), p.head_dim, dtype=k.dtype, device=dev)
+    v_out = torch.empty(max(cap, 1), p.head_dim, dtype=v.dtype, device=dev)
+    units = p.num_seqs * p.num_kv_heads
+    lengths = torch.zeros(units, dtype=torch.int32, device=dev)
+    offsets = torch.zeros(units + 1, dtype=torch.int64, device=dev)
+    kept = torch.empty(max(cap, 1), dtype=torch.int32, device=dev) if want_kept_idx else None
+    scores = torch.empty(p.num_kv_heads, total_tokens, dtype=torch.float32, device=dev) if want_scores else None
+    if workspace is None:
+        workspace = torch.empty(refree_workspace_size(p, total_tokens), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    refree_compress_layer(p, q_win, k, v, seq_start, seq_len, total_tokens, k_out, v_out, cap, lengths, offsets,
+                          kept, scores, workspace, status, stream)
+    return LayerResult(k_out, v_out, lengths.view(p.num_seqs, p.num_kv_heads), offsets, kept, scores, status)

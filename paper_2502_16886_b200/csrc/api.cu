@@ -1,0 +1,298 @@
+// C-ABI entry points: argument checks, workspace layout, launch sequences.
+#include <string.h>
+
+#include "refree_internal.cuh"
+
+namespace refree {
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
+{
+    Workspace w;
+    const int64_t U = (int64_t)p.num_seqs * p.num_kv_heads;
+    const int64_t G = p.num_q_heads / p.num_kv_heads;
+    const int64_t rows = G * p.window;
+    const int64_t tiles = total_tokens / kTile + p.num_seqs;
+    size_t off = 0;
+    w.part_off = off;   w.part_bytes = align256((size_t)(tiles * p.num_kv_heads * rows) * sizeof(float2)); off += w.part_bytes;
+    w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows) * sizeof(float));                        off += w.lse_bytes;
+    w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
+    w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
+    w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
+    w.kept_off = off;   w.kept_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(int32_t)); off += w.kept_bytes;
+    w.total = off;
+    return w;
+}
+
+static refree_status check_params(const refree_params *p, int64_t total_tokens)
+{
+    if (!p) return REFREE_ERR_INVALID_ARG;
+    if (p->num_seqs < 1 || p->num_q_heads < 1 || p->num_kv_heads < 1) return REFREE_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads != 0) return REFREE_ERR_INVALID_ARG;
+    if (p->window < 1 || p->sink < 0) return REFREE_ERR_INVALID_ARG;
+    if (!(p->threshold >= 0.0f && p->threshold < 1.0f)) return REFREE_ERR_INVALID_ARG;
+    if (p->rank_mode != REFREE_RANK_POSITION && p->rank_mode != REFREE_RANK_SCORE) return REFREE_ERR_INVALID_ARG;
+    if (p->scope != REFREE_SCOPE_HEAD && p->scope != REFREE_SCOPE_LAYER) return REFREE_ERR_INVALID_ARG;
+    if (p->dtype != REFREE_DTYPE_F32 && p->dtype != REFREE_DTYPE_BF16) return REFREE_ERR_INVALID_ARG;
+    if (total_tokens < 0 || total_tokens > 0x7fffffffLL - kTile) return REFREE_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return REFREE_ERR_UNSUPPORTED;
+    if (p->num_seqs > kMaxSeqs) return REFREE_ERR_UNSUPPORTED;
+    if ((int64_t)p->num_seqs * p->num_kv_heads > 65535) return REFREE_ERR_UNSUPPORTED;
+    if ((int64_t)(p->num_q_heads / p->num_kv_heads) * p->window > kMaxRows) return REFREE_ERR_UNSUPPORTED;
+    return REFREE_OK;
+}
+
+static refree_status check_kv_layout(const refree_params *p, const void *k, const void *v, bool need_v)
+{
+    const int esz = p->dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    if (p->kv_tokens < 0) return REFREE_ERR_INVALID_ARG;
+    if (p->k_stride_tok < p->head_dim || p->k_stride_seq < 0 || p->k_stride_head < 0) return REFREE_ERR_INVALID_ARG;
+    // 16-byte vector access to every row
+    if ((reinterpret_cast<uintptr_t>(k) & 15) || (p->k_stride_tok * esz) % 16 || (p->k_stride_head * esz) % 16 ||
+        (p->k_stride_seq * esz) % 16)
+        return REFREE_ERR_UNSUPPORTED;
+    if (need_v) {
+        if (p->v_stride_tok < p->head_dim || p->v_stride_seq < 0 || p->v_stride_head < 0) return REFREE_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(v) & 15) || (p->v_stride_tok * esz) % 16 || (p->v_stride_head * esz) % 16 ||
+            (p->v_stride_seq * esz) % 16)
+            return REFREE_ERR_UNSUPPORTED;
+    }
+    return REFREE_OK;
+}
+
+static refree_status from_cuda(cudaError_t e) { return e == cudaSuccess ? REFREE_OK : REFREE_ERR_CUDA; }
+
+static cudaError_t run_score(const refree_params &p, const void *q_win, const void *k,
+                             const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                             float *scores, char *ws, const Workspace &lay, int32_t *dev_status,
+                             cudaStream_t st)
+{
+    if (score_tc_supported(p))
+        return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
+    return launch_score_generic(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
+}
+
+}  // namespace refree
+
+using namespace refree;
+
+extern "C" {
+
+void refree_default_params(refree_params *p)
+{
+    if (!p) return;
+    memset(p, 0, sizeof(*p));
+    p->window = 1;
+    p->sink = 4;
+    p->threshold = 0.01f;
+    p->rank_mode = REFREE_RANK_POSITION;
+    p->scope = REFREE_SCOPE_HEAD;
+    p->keep_window = 1;
+    p->force_full = 0;
+    p->dtype = REFREE_DTYPE_BF16;
+}
+
+const char *refree_status_string(refree_status s)
+{
+    switch (s) {
+    case REFREE_OK: return "ok";
+    case REFREE_ERR_INVALID_ARG: return "invalid argument";
+    case REFREE_ERR_UNSUPPORTED: return "unsupported shape, type or alignment";
+    case REFREE_ERR_WORKSPACE: return "workspace missing or too small";
+    case REFREE_ERR_CAPACITY: return "output capacity too small";
+    case REFREE_ERR_CUDA: return "CUDA runtime error";
+    case REFREE_ERR_TIMEOUT: return "a bounded on-device wait gave up";
+    case REFREE_ERR_NONFINITE: return "non-finite score";
+    }
+    return "unknown status";
+}
+
+refree_status refree_workspace_size(const refree_params *p, int64_t total_tokens, size_t *bytes)
+{
+    if (!bytes) return REFREE_ERR_INVALID_ARG;
+    const refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    *bytes = workspace_layout(*p, total_tokens).total;
+    return REFREE_OK;
+}
+
+refree_status refree_score(const refree_params *p, const void *q_win, const void *k,
+                           const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                           float *scores, void *workspace, size_t workspace_bytes,
+                           int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    if (!q_win || !k || !seq_start || !seq_len || !scores) return REFREE_ERR_INVALID_ARG;
+    st = check_kv_layout(p, k, nullptr, false);
+    if (st != REFREE_OK) return st;
+    const Workspace lay = workspace_layout(*p, total_tokens);
+    if (!workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    if (total_tokens == 0) return REFREE_OK;
+    return from_cuda(run_score(*p, q_win, k, seq_start, seq_len, total_tokens, scores, (char *)workspace, lay,
+                               device_status, (cudaStream_t)stream));
+}
+
+refree_status refree_select_budget(const refree_params *p, const float *scores,
+                                   const int32_t *seq_len, int64_t total_tokens,
+                                   int32_t *lengths, int64_t *offsets,
+                                   int32_t *kept_idx, int64_t capacity_rows,
+                                   void *workspace, size_t workspace_bytes,
+                                   int32_t *device_status, void *stream)
+{
+    const refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    if (!scores || !seq_len || !lengths || !offsets || capacity_rows < 0) return REFREE_ERR_INVALID_ARG;
+    const Workspace lay = workspace_layout(*p, total_tokens);
+    if (!workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    return from_cuda(launch_select(*p, scores, seq_len, total_tokens, lengths, offsets, kept_idx, capacity_rows,
+                                   (char *)workspace, lay, device_status, (cudaStream_t)stream));
+}
+
+refree_status refree_compact(const refree_params *p, const void *k, const void *v,
+                             const int32_t *seq_start, const int32_t *seq_len,
+                             const int32_t *lengths, const int64_t *offsets,
+                             const int32_t *kept_idx, void *k_out, void *v_out,
+                             int64_t capacity_rows, int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, 0);
+    if (st != REFREE_OK) return st;
+    if (!k || !v || !seq_start || !seq_len || !lengths || !offsets || !kept_idx || !k_out || !v_out ||
+        capacity_rows < 0)
+        return REFREE_ERR_INVALID_ARG;
+    st = check_kv_layout(p, k, v, true);
+    if (st != REFREE_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
+        return REFREE_ERR_UNSUPPORTED;
+    return from_cuda(launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept_idx, false, k_out, v_out,
+                                    capacity_rows, device_status, (cudaStream_t)stream));
+}
+
+refree_status refree_compress_layer(const refree_params *p, const void *q_win,
+                                    const void *k, const void *v,
+                                    const int32_t *seq_start, const int32_t *seq_len,
+                                    int64_t total_tokens,
+                                    void *k_out, void *v_out, int64_t capacity_rows,
+                                    int32_t *lengths, int64_t *offsets,
+                                    int32_t *kept_idx, float *scores,
+                                    void *workspace, size_t workspace_bytes,
+                                    int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    if (!q_win || !k || !v || !seq_start || !seq_len || !k_out || !v_out || !lengths || !offsets ||
+        capacity_rows < 0)
+        return REFREE_ERR_INVALID_ARG;
+    st = check_kv_layout(p, k, v, true);
+    if (st != REFREE_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
+        return REFREE_ERR_UNSUPPORTED;
+    const Workspace lay = workspace_layout(*p, total_tokens);
+    if (!workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    char *ws = (char *)workspace;
+    cudaStream_t cs = (cudaStream_t)stream;
+    float *sc = scores ? scores : reinterpret_cast<float *>(ws + lay.scores_off);
+    const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
+    int32_t *kept = kept_idx ? kept_idx : (ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off));
+    cudaError_t e = cudaSuccess;
+    // a frozen layer needs no scores unless the caller asked for them
+    if (total_tokens > 0 && (!p->force_full || scores))
+        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, k_out, v_out, capacity_rows,
+                       device_status, cs);
+    return from_cuda(e);
+}
+
+refree_status refree_host_arena_size(const refree_params *p, int64_t total_tokens,
+                                     int64_t kv_elems, int64_t capacity_rows, size_t *bytes)
+{
+    if (!bytes || kv_elems < 0 || capacity_rows < 0) return REFREE_ERR_INVALID_ARG;
+    const refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    const size_t esz = p->dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const size_t U = (size_t)p->num_seqs * p->num_kv_heads;
+    size_t tot = 0;
+    tot += align256((size_t)p->num_seqs * p->num_q_heads * p->window * p->head_dim * esz);  // q_win
+    tot += 2 * align256((size_t)kv_elems * esz);                                            // k, v
+    tot += 2 * align256((size_t)p->num_seqs * sizeof(int32_t));                             // seq_start, seq_len
+    tot += 2 * align256((size_t)capacity_rows * p->head_dim * esz);                         // k_out, v_out
+    tot += align256(U * sizeof(int32_t)) + align256((U + 1) * sizeof(int64_t));             // lengths, offsets
+    tot += align256((size_t)capacity_rows * sizeof(int32_t));                               // kept_idx
+    tot += align256((size_t)p->num_kv_heads * total_tokens * sizeof(float));                // scores
+    tot += align256(sizeof(int32_t));                                                       // device status
+    tot += workspace_layout(*p, total_tokens).total;
+    *bytes = tot;
+    return REFREE_OK;
+}
+
+refree_status refree_compress_layer_host(const refree_params *p, const void *q_win,
+                                         const void *k, const void *v, int64_t kv_elems,
+                                         const int32_t *seq_start, const int32_t *seq_len,
+                                         int64_t total_tokens,
+                                         void *k_out, void *v_out, int64_t capacity_rows,
+                                         int32_t *lengths, int64_t *offsets,
+                                         int32_t *kept_idx, float *scores,
+                                         void *arena, size_t arena_bytes, void *stream)
+{
+    size_t need = 0;
+    refree_status st = refree_host_arena_size(p, total_tokens, kv_elems, capacity_rows, &need);
+    if (st != REFREE_OK) return st;
+    if (!q_win || !k || !v || !seq_start || !seq_len || !k_out || !v_out || !lengths || !offsets)
+        return REFREE_ERR_INVALID_ARG;
+    if (!arena || arena_bytes < need || (reinterpret_cast<uintptr_t>(arena) & 255)) return REFREE_ERR_WORKSPACE;
+    cudaStream_t cs = (cudaStream_t)stream;
+    const size_t esz = p->dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const size_t U = (size_t)p->num_seqs * p->num_kv_heads;
+    char *a = (char *)arena;
+    auto take = [&](size_t bytes) { char *r = a; a += align256(bytes); return r; };
+    const size_t q_bytes = (size_t)p->num_seqs * p->num_q_heads * p->window * p->head_dim * esz;
+    const size_t kv_bytes = (size_t)kv_elems * esz;
+    const size_t row_bytes = (size_t)p->head_dim * esz;
+    char *d_q = take(q_bytes), *d_k = take(kv_bytes), *d_v = take(kv_bytes);
+    int32_t *d_start = (int32_t *)take(p->num_seqs * sizeof(int32_t));
+    int32_t *d_len = (int32_t *)take(p->num_seqs * sizeof(int32_t));
+    char *d_ko = take(capacity_rows * row_bytes), *d_vo = take(capacity_rows * row_bytes);
+    int32_t *d_lengths = (int32_t *)take(U * sizeof(int32_t));
+    int64_t *d_offsets = (int64_t *)take((U + 1) * sizeof(int64_t));
+    int32_t *d_kept = (int32_t *)take((size_t)capacity_rows * sizeof(int32_t));
+    float *d_scores = (float *)take((size_t)p->num_kv_heads * total_tokens * sizeof(float));
+    int32_t *d_status = (int32_t *)take(sizeof(int32_t));
+    char *d_ws = a;
+    const size_t ws_bytes = workspace_layout(*p, total_tokens).total;
+
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d_q, q_win, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if ((e = cudaMemcpyAsync(d_k, k, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if ((e = cudaMemcpyAsync(d_v, v, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if ((e = cudaMemcpyAsync(d_start, seq_start, p->num_seqs * sizeof(int32_t), cudaMemcpyHostToDevice, cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if ((e = cudaMemcpyAsync(d_len, seq_len, p->num_seqs * sizeof(int32_t), cudaMemcpyHostToDevice, cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if ((e = cudaMemsetAsync(d_status, 0, sizeof(int32_t), cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    st = refree_compress_layer(p, d_q, d_k, d_v, d_start, d_len, total_tokens, d_ko, d_vo, capacity_rows,
+                               d_lengths, d_offsets, kept_idx ? d_kept : nullptr, scores ? d_scores : nullptr,
+                               d_ws, ws_bytes, d_status, stream);
+    if (st != REFREE_OK) return st;
+    int32_t h_status = 0;
+    cudaMemcpyAsync(lengths, d_lengths, U * sizeof(int32_t), cudaMemcpyDeviceToHost, cs);
+    cudaMemcpyAsync(offsets, d_offsets, (U + 1) * sizeof(int64_t), cudaMemcpyDeviceToHost, cs);
+    cudaMemcpyAsync(&h_status, d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, cs);
+    if ((e = cudaStreamSynchronize(cs)) != cudaSuccess) return REFREE_ERR_CUDA;
+    if (h_status & REFREE_DEV_TIMEOUT) return REFREE_ERR_TIMEOUT;
+    if (h_status & REFREE_DEV_CAPACITY) return REFREE_ERR_CAPACITY;
+    if (h_status & REFREE_DEV_NONFINITE) return REFREE_ERR_NONFINITE;
+    const int64_t rows = offsets[U];
+    cudaMemcpyAsync(k_out, d_ko, (size_t)rows * row_bytes, cudaMemcpyDeviceToHost, cs);
+    cudaMemcpyAsync(v_out, d_vo, (size_t)rows * row_bytes, cudaMemcpyDeviceToHost, cs);
+    if (kept_idx) cudaMemcpyAsync(kept_idx, d_kept, (size_t)rows * sizeof(int32_t), cudaMemcpyDeviceToHost, cs);
+    if (scores)
+        cudaMemcpyAsync(scores, d_scores, (size_t)p->num_kv_heads * total_tokens * sizeof(float), cudaMemcpyDeviceToHost, cs);
+    return from_cuda(cudaStreamSynchronize(cs));
+}
+
+}  // extern "C"

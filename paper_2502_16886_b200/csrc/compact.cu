@@ -1,0 +1,94 @@
+// Step S7: gather the kept K and V rows of every unit into the dense ragged
+// output (Algorithm 1, "Compress" steps).  Pure data movement: 16-byte vector
+// loads and stores, several rows in flight per thread.  Rows are copied bit for
+// bit.  With position ranking the kept set is two contiguous ranges, so the
+// source row follows from (b, m, n) and no index list is read.
+#include "refree_internal.cuh"
+
+namespace refree {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;
+
+__device__ inline int4 ld_stream(const int4 *p)
+{
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ inline void st_stream(int4 *p, const int4 &v)
+{
+    asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads)
+compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq_start,
+               const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
+               const int32_t *kept_idx, int position_ranges, char *k_out, char *v_out,
+               int64_t capacity_rows, int32_t *dev_status)
+{
+    const int Hkv = p.num_kv_heads;
+    const int u = blockIdx.y, s = u / Hkv, g = u % Hkv;
+    const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const int row_bytes = p.head_dim * esz;
+    const int vec_per_row = row_bytes >> 4;
+    const int vshift = 31 - __clz(vec_per_row);
+    const int n = max(seq_len[s], 0);
+    const int b = lengths[u];
+    const int64_t off = offsets[u];
+    if (b < 0 || b > n || off < 0 || off + b > capacity_rows) {
+        if (threadIdx.x == 0 && blockIdx.x == 0 && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
+        return;
+    }
+    const int head = min(b, min(p.sink, n));
+    const int64_t tok0 = seq_start[s];
+    const char *kb = k + ((int64_t)s * p.k_stride_seq + tok0 * p.k_stride_tok + (int64_t)g * p.k_stride_head) * esz;
+    const char *vb = v + ((int64_t)s * p.v_stride_seq + tok0 * p.v_stride_tok + (int64_t)g * p.v_stride_head) * esz;
+    const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
+    char *ko = k_out + off * row_bytes, *vo = v_out + off * row_bytes;
+    const int32_t *idx = kept_idx ? kept_idx + off : nullptr;
+    const int64_t nvec = (int64_t)b << vshift;
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    for (int64_t e0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; e0 < nvec; e0 += stride * kUnroll) {
+        int4 kv[kUnroll], vv[kUnroll];
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r) {
+            const int64_t e = e0 + r * stride;
+            if (e < nvec) {
+                const int t = (int)(e >> vshift), c = (int)(e & (vec_per_row - 1));
+                const int src = position_ranges ? (t < head ? t : n - b + t) : idx[t];
+                kv[r] = *reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok + c * 16);
+                vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16));
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r) {
+            const int64_t e = e0 + r * stride;
+            if (e < nvec) {
+                st_stream(reinterpret_cast<int4 *>(ko + e * 16), kv[r]);
+                st_stream(reinterpret_cast<int4 *>(vo + e * 16), vv[r]);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
+                           const int32_t *seq_start, const int32_t *seq_len,
+                           const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
+                           bool position_ranges, void *k_out, void *v_out, int64_t capacity_rows,
+                           int32_t *dev_status, cudaStream_t st)
+{
+    const int U = p.num_seqs * p.num_kv_heads;
+    const int gx = max(1, (148 * 8) / U);
+    compact_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
+                                                     lengths, offsets, kept_idx, position_ranges ? 1 : 0,
+                                                     (char *)k_out, (char *)v_out, capacity_rows, dev_status);
+    return cudaGetLastError();
+}
+
+}  // namespace refree

@@ -1,0 +1,110 @@
+// Internal declarations shared by the kernels of the compression-pass library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "refreekv.h"
+
+namespace refree {
+
+constexpr int kMaxSeqs = 1024;   // sequences per call (prefix tables live in shared memory)
+constexpr int kTile = 128;       // positions per scoring tile
+constexpr int kMaxRows = 1024;   // G * window handled by the generic scoring path
+
+// Bounded spin: polls before a wait gives up and reports REFREE_DEV_TIMEOUT.
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// Layout of the caller-provided workspace.  All offsets are multiples of 256.
+struct Workspace {
+    size_t part_off, part_bytes;       // per (tile, head, row) softmax partials (float2: max, sum)
+    size_t lse_off, lse_bytes;         // per (unit, row) log2-sum-exp of the row's logits
+    size_t cnt_off, cnt_bytes;         // per unit arrival counters (zeroed by each call)
+    size_t cut_off, cut_bytes;         // per unit selection result (struct Cut)
+    size_t scores_off, scores_bytes;   // scratch scores when the caller passes none
+    size_t kept_off, kept_bytes;       // scratch kept_idx when the caller passes none
+    size_t total;
+};
+
+// Result of the stopping rule for one unit, enough to enumerate its kept set.
+//   position ranking: kept = [0, min(b, lead)) U [n - (b - lead), n)
+//   score ranking:    kept = the first min(b, lead + w_eff) protected positions in
+//                     order (leading then window), plus unprotected positions whose
+//                     key is above `tau`, plus the first `ties` (by position) whose
+//                     key equals `tau`.
+struct Cut {
+    int32_t b;          // budget (kept count)
+    int32_t ties;       // score ranking: number of positions with key == tau to keep
+    uint64_t tau;       // score ranking: key threshold (bits of the fp64 squared score)
+    int32_t prot_kept;  // score ranking: protected positions kept
+    int32_t pad;
+};
+
+Workspace workspace_layout(const refree_params &p, int64_t total_tokens);
+
+inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Per-CTA tables: running sums of sequence lengths and of tiles per sequence.
+struct SeqTables {
+    int32_t pack[kMaxSeqs + 1];   // positions before sequence s in the packed score array
+    int32_t tiles[kMaxSeqs + 1];  // scoring tiles before sequence s
+};
+
+__device__ inline void build_seq_tables(SeqTables &t, const int32_t *seq_len, int B)
+{
+    if (threadIdx.x == 0) {
+        int32_t a = 0, b = 0;
+        for (int s = 0; s < B; ++s) {
+            t.pack[s] = a;
+            t.tiles[s] = b;
+            const int n = max(seq_len[s], 0);
+            a += n;
+            b += ceil_div(n, kTile);
+        }
+        t.pack[B] = a;
+        t.tiles[B] = b;
+    }
+    __syncthreads();
+}
+
+// Largest s with table[s] <= x (table ascending, table[0] == 0).
+__device__ inline int find_seq(const int32_t *table, int B, int x)
+{
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (table[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <typename T> __device__ inline float to_float(T v);
+template <> __device__ inline float to_float<float>(float v) { return v; }
+template <> __device__ inline float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// ---- launchers (defined in the .cu files) ----------------------------------
+cudaError_t launch_score_generic(const refree_params &p, const void *q_win, const void *k,
+                                 const int32_t *seq_start, const int32_t *seq_len,
+                                 int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
+                                 int32_t *dev_status, cudaStream_t st);
+
+// Returns false when the shape is outside what the tensor-core path handles.
+bool score_tc_supported(const refree_params &p);
+cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
+                            const int32_t *seq_start, const int32_t *seq_len,
+                            int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
+                            int32_t *dev_status, cudaStream_t st);
+
+cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
+                          int64_t total_tokens, int32_t *lengths, int64_t *offsets,
+                          int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,
+                          int32_t *dev_status, cudaStream_t st);
+
+cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
+                           const int32_t *seq_start, const int32_t *seq_len,
+                           const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
+                           bool position_ranges, void *k_out, void *v_out, int64_t capacity_rows,
+                           int32_t *dev_status, cudaStream_t st);
+
+}  // namespace refree

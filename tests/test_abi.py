@@ -1,0 +1,76 @@
+"""The C-ABI library builds, loads and exports every entry point the header
+declares; host-side argument checks answer without touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2502_16886_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def declared_functions():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(refree_[a-z_0-9]+)\s*\(", text))
+    return names
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    names = declared_functions()
+    assert {"refree_score", "refree_select_budget", "refree_compact", "refree_compress_layer"} <= names
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in include/ but not exported"
+        assert name in binding.SIGNATURES, f"{name} has no binding"
+
+
+def test_status_strings_and_defaults(lib):
+    assert binding.status_string(0) == "ok"
+    assert len({binding.status_string(c) for c in range(8)}) == 8
+    d = binding.default_params()
+    assert (d.window, d.sink, d.rank_mode, d.scope, d.keep_window, d.force_full, d.dtype) == (1, 4, 0, 0, 1, 0, 1)
+    assert abs(d.threshold - 0.01) < 1e-9
+
+
+def test_params_struct_matches_header_layout(lib):
+    # 12 int32/float fields, then 7 int64
+    assert ctypes.sizeof(binding.CParams) == 12 * 4 + 7 * 8
+
+
+def test_host_side_validation_needs_no_gpu(lib):
+    good = binding.Params(1, 4, 2, 64, window=8, kv_tokens=128, k_strides=(0, 64, 8192), v_strides=(0, 64, 8192))
+    assert binding.refree_workspace_size(good, 128) > 0
+    for field, val, code in [("num_q_heads", 3, 1), ("window", 0, 1), ("threshold", 1.0, 1), ("threshold", -0.1, 1),
+                             ("head_dim", 96, 2), ("rank_mode", 5, 1), ("dtype", 9, 1), ("num_seqs", 5000, 2)]:
+        bad = binding.Params(**{**good.__dict__, field: val})
+        with pytest.raises(binding.RefreeError) as ei:
+            binding.refree_workspace_size(bad, 128)
+        assert ei.value.code == code
+    # null pointers and a missing workspace are caught before any launch
+    c = good.c_struct()
+    rc = lib.refree_score(ctypes.byref(c), None, None, None, None, 128, None, None, 0, None, None)
+    assert rc == 1
+    fake = ctypes.c_void_p(4096)
+    rc = lib.refree_score(ctypes.byref(c), fake, fake, fake, fake, 128, fake, None, 0, None, None)
+    assert rc == 3
+    rc = lib.refree_score(ctypes.byref(c), fake, ctypes.c_void_p(4100), fake, fake, 128, fake, fake, 1 << 30, None, None)
+    assert rc == 2          # K not 16-byte aligned
+
+
+def test_missing_library_is_an_error(monkeypatch, lib):
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/librefreekv.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.lib()

@@ -157,6 +157,10 @@ refree_status refree_compress_layer_host(const refree_params *p, const void *q_w
                                          int32_t *kept_idx, float *scores,
                                          void *arena, size_t arena_bytes, void *stream);
 
+/* Diagnostic with no counterpart in the paper: the number of CUDA kernels this
+ * library has enqueued in this process so far (all entry points, all streams). */
+int64_t refree_kernel_launch_count(void);
+
 /* Static string for a status code. */
 const char *refree_status_string(refree_status s);
 

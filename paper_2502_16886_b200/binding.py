@@ -77,6 +77,7 @@ _PP = ctypes.POINTER(CParams)
 SIGNATURES = {
     "refree_default_params": (None, [_PP]),
     "refree_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "refree_kernel_launch_count": (ctypes.c_int64, []),
     "refree_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
     "refree_score": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
     "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
@@ -107,6 +108,10 @@ def lib():
 
 def status_string(code: int) -> str:
     return lib().refree_status_string(int(code)).decode()
+
+
+def refree_kernel_launch_count() -> int:
+    return int(lib().refree_kernel_launch_count())
 
 
 def default_params() -> CParams:

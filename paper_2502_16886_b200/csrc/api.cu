@@ -1,9 +1,14 @@
 // C-ABI entry points: argument checks, workspace layout, launch sequences.
 #include <string.h>
 
+#include <atomic>
+
 #include "refree_internal.cuh"
 
 namespace refree {
+
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -92,6 +97,8 @@ void refree_default_params(refree_params *p)
     p->force_full = 0;
     p->dtype = REFREE_DTYPE_BF16;
 }
+
+int64_t refree_kernel_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char *refree_status_string(refree_status s)
 {

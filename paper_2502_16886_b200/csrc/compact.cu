@@ -88,6 +88,7 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
     compact_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
                                                      lengths, offsets, kept_idx, position_ranges ? 1 : 0,
                                                      (char *)k_out, (char *)v_out, capacity_rows, dev_status);
+    count_launches(1);
     return cudaGetLastError();
 }
 

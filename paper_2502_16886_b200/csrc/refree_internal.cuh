@@ -43,6 +43,9 @@ struct Cut {
 
 Workspace workspace_layout(const refree_params &p, int64_t total_tokens);
 
+// Bookkeeping for refree_kernel_launch_count(): every launcher adds the kernels it enqueued.
+void count_launches(int n);
+
 inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Per-CTA tables: running sums of sequence lengths and of tiles per sequence.

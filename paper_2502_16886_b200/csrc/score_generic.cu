@@ -211,6 +211,7 @@ cudaError_t run(const refree_params &p, const void *q_win, const void *k, const 
     score_combine_generic<<<(int)std::min<int64_t>((rows + 255) / 256, 1024), 256, 0, st>>>(p, seq_len, part, lse);
     score_colsum_generic<T, D><<<grid, kThreads, smem, st>>>(p, (const T *)q_win, (const T *)k, seq_start, seq_len,
                                                             lse, total_tokens, scores, dev_status);
+    count_launches(3);
     return cudaGetLastError();
 }
 

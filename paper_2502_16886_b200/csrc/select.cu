@@ -360,6 +360,7 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     }
     emit_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, offsets,
                                                   kept_idx, capacity_rows, dev_status);
+    count_launches(2);
     return cudaGetLastError();
 }
 

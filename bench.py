@@ -1,0 +1,461 @@
+#!/usr/bin/env python
+"""Benchmark of the post-prefill KV-compression pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+                    [--rank-mode position|score] [--impl ours|reference]
+
+One step = the fused pass (refree_compress_layer: score, select, compact) over
+every layer of one synthetic prefill cache that is already resident in HBM.
+Prints ONE JSON line on rank 0.  With N > 1 (launched by torchrun) every rank
+runs its own replica of the workload: the units of the pass are independent, so
+there is no collective on the data path (weak scaling).
+
+`--impl reference` times the CPU oracle on the host cores instead (a bounded
+sample of the same workload per step); it exists to put a number beside the
+GPU's, not as a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "kv_tokens_compressed_per_sec_per_layer"
+UNIT = "tokens/s/layer"
+DEFAULT_WORKLOAD = "mistral7b_32k"      # the 32K-token, 32q/8kv, d=128 cache the target is quoted on
+FALLBACK_HBM_GBS = 6650.0
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+# ----------------------------------------------------------- distributed ----
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), \
+        int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def dist_setup(backend: str):
+    """Join the process group when launched with WORLD_SIZE > 1."""
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, local_rank, world
+
+
+def dist_barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def dist_max(value: float, world: int, device) -> float:
+    """Max over ranks of a host float (the job time is the slowest rank's)."""
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def dist_sum(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def aggregate_throughput(tokens_per_rank: float, ms_per_step_max: float, layers: int, world_tokens: float) -> float:
+    """Whole-job tokens/s per layer: tokens all ranks processed in a layer pass / slowest rank's layer time."""
+    del tokens_per_rank
+    return world_tokens / (ms_per_step_max * 1e-3 / layers)
+
+
+# ------------------------------------------------------------- clocks ----
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False).name
+        self.proc = None
+        self.gpu = gpu_index
+        self.t0 = self.t1 = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu=timestamp,{self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        import datetime
+        rows = []
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
+            except ValueError:
+                continue
+        os.unlink(self.path)
+        inside = [r for r in rows if self.t0 is not None and self.t0 - 0.05 <= r[0] <= self.t1 + 0.05]
+        use = inside if inside else rows[-3:]
+        if not use:
+            return out
+        out["sm_mhz"] = statistics.median(r[1] for r in use)
+        out["sm_max_mhz"] = use[0][2]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        out["reasons"] = [n for i, n in enumerate(names) if any(r[3][i].lower().startswith("active") for r in use)]
+        out["samples"] = len(inside)
+        return out
+
+
+# ------------------------------------------------------------ workload ----
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(cfg, seq_lens, lengths):
+    """Bytes the pass must move for one layer: K read once for scoring, kept V
+    read, kept K and V written, fp32 scores written (the kept-K re-read is
+    assumed served from L2).  Returns (1+3rho) form and the (1+4rho) form."""
+    row = cfg.head_dim * cfg.elem_bytes
+    a = b4 = 0
+    for s, n in enumerate(seq_lens):
+        for g in range(cfg.num_kv_heads):
+            kept = int(lengths[s][g])
+            a += n * row + 3 * kept * row + 4 * n
+            b4 += n * row + 4 * kept * row + 4 * n
+    return a, b4
+
+
+def run_ours(args):
+    from paper_2502_16886_b200 import binding, build, workloads
+    rank, local_rank, world = dist_setup("nccl")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    build.build()
+    binding.lib()
+    cfg = workloads.get_config(args.workload)
+    L = args.layers or cfg.num_layers
+    rank_mode = binding.RANK_SCORE if args.rank_mode == "score" else binding.RANK_POSITION
+    seq_lens = workloads.sequence_lengths(cfg)
+    total = sum(seq_lens)
+    cap = cfg.num_kv_heads * total
+    units = len(seq_lens) * cfg.num_kv_heads
+
+    t0 = time.time()
+    layers = []
+    params = None
+    for l in range(L):
+        lay = workloads.make_layer(cfg, l)
+        if params is None:
+            params = binding.params_for(cfg, lay, rank_mode=rank_mode)
+        layers.append(dict(
+            q=lay.q_win.to(dev), k=lay.k.to(dev), v=lay.v.to(dev),
+            k_out=torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype, device=dev),
+            v_out=torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype, device=dev),
+            lengths=torch.zeros(units, dtype=torch.int32, device=dev),
+            offsets=torch.zeros(units + 1, dtype=torch.int64, device=dev)))
+        if l == 0:
+            host0 = lay
+    seq_start = host0.seq_start.to(dev)
+    seq_len = host0.seq_len.to(dev)
+    ws = torch.empty(binding.refree_workspace_size(params, total), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    if rank == 0:
+        log(f"[bench] {cfg.name}: {L} layers generated in {time.time() - t0:.1f}s, "
+            f"{torch.cuda.memory_allocated(dev) / 2**30:.1f} GiB on device")
+
+    def one_layer(d):
+        binding.refree_compress_layer(params, d["q"], d["k"], d["v"], seq_start, seq_len, total, d["k_out"],
+                                      d["v_out"], cap, d["lengths"], d["offsets"], None, None, ws, status)
+
+    def step():
+        for d in layers:
+            one_layer(d)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    dist_barrier(world)
+    torch.cuda.synchronize()
+    launches0 = binding.refree_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_begin()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    sampler.mark_end()
+    dist_barrier(world)
+    launches = binding.refree_kernel_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_step = dist_max(ev0.elapsed_time(ev1) / args.steps, world, dev)
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    value = aggregate_throughput(total, ms_step, L, dist_sum(float(total), world, dev))
+
+    if rank != 0:
+        if world > 1:
+            dist_barrier(world)
+        return
+
+    # kept ratio and algorithmic bytes, from the budgets the timed steps produced
+    all_lengths = [d["lengths"].view(len(seq_lens), cfg.num_kv_heads).cpu().tolist() for d in layers]
+    rho = sum(sum(map(sum, ln)) for ln in all_lengths) / (L * cfg.num_kv_heads * total)
+    bytes3 = sum(algorithmic_bytes(cfg, seq_lens, ln)[0] for ln in all_lengths) / L
+    bytes4 = sum(algorithmic_bytes(cfg, seq_lens, ln)[1] for ln in all_lengths) / L
+    peak, peak_kind = hbm_peak()
+    ms_layer = ms_step / L
+    pass_gbs = bytes3 / (ms_layer * 1e-3) / 1e9
+
+    # per-stage device times, one event-bracketed sweep over the layers through the stage entry points
+    scores = torch.empty(cfg.num_kv_heads, total, dtype=torch.float32, device=dev)
+    kept = torch.empty(cap, dtype=torch.int32, device=dev)
+    stage_ms = {"score": 0.0, "select": 0.0, "compact": 0.0}
+    reps = 3
+    for rep in range(reps + 1):
+        for d in layers:
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record()
+            binding.refree_score(params, d["q"], d["k"], seq_start, seq_len, total, scores, ws, status)
+            e[1].record()
+            binding.refree_select_budget(params, scores, seq_len, total, d["lengths"], d["offsets"], kept, cap, ws, status)
+            e[2].record()
+            binding.refree_compact(params, d["k"], d["v"], seq_start, seq_len, d["lengths"], d["offsets"], kept,
+                                   d["k_out"], d["v_out"], cap, status)
+            e[3].record()
+            torch.cuda.synchronize()
+            if rep > 0:
+                for i, name in enumerate(stage_ms):
+                    stage_ms[name] += e[i].elapsed_time(e[i + 1]) / (reps * L)
+    row = cfg.head_dim * cfg.elem_bytes
+    kept_rows = rho * cfg.num_kv_heads * total
+    stage_bytes = {"score": cfg.num_kv_heads * total * (row + 4), "select": cfg.num_kv_heads * total * 8,
+                   "compact": 4 * kept_rows * row + 4 * kept_rows}
+    dominant = max(stage_ms, key=stage_ms.get)
+    dom_gbs = stage_bytes[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
+    roofline = {"kernel": f"refree_{dominant} stage", "bound": "hbm", "achieved": round(dom_gbs, 1),
+                "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(dom_gbs / peak, 4),
+                "traffic": None, "bytes_per_launch": int(stage_bytes[dominant]),
+                "ms_per_launch": round(stage_ms[dominant], 5),
+                "stages_ms": {k: round(v, 5) for k, v in stage_ms.items()},
+                "stages_gbs": {k: round(stage_bytes[k] / (stage_ms[k] * 1e-3) / 1e9, 1) for k in stage_ms}}
+    roofline_pass = {"bound": "hbm", "achieved": round(pass_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}",
+                     "unit": "GB/s", "frac": round(pass_gbs / peak, 4), "frac_of_8TBps": round(pass_gbs / 8000.0, 4),
+                     "bytes_per_layer": int(bytes3), "bytes_per_layer_with_kept_k_reread": int(bytes4),
+                     "kept_ratio": round(rho, 4), "ms_per_layer": round(ms_layer, 5)}
+
+    e2e = measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args)
+    cpu_baseline = measure_cpu_baseline(cfg, rank_mode, total, args) if world == 1 and not args.no_cpu_baseline else None
+
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.num_q_heads, "kv_heads": cfg.num_kv_heads,
+                   "head_dim": cfg.head_dim, "seq_lens": seq_lens if len(seq_lens) <= 8 else len(seq_lens),
+                   "window": cfg.window, "sink": cfg.sink, "threshold": 0.01, "rank_mode": args.rank_mode,
+                   "scope": "head", "layout": "head_major",
+                   "l2": f"each step sweeps {L} layers of distinct K/V buffers "
+                         f"({L * 2 * cfg.num_kv_heads * total * row / 2**30:.1f} GiB), larger than L2",
+                   "replicas": world},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
+        "roofline": roofline, "roofline_pass": roofline_pass, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist_barrier(world)
+
+
+def measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args):
+    """Same metric through the host-buffer entry point: pinned host inputs are
+    copied in, the pass runs, kept rows and budgets are copied back, every layer."""
+    n_lay = min(L, 4)
+    row = cfg.head_dim * cfg.elem_bytes
+    host = []
+    for l in range(n_lay):
+        lay = workloads.make_layer(cfg, l)
+        host.append(dict(q=lay.q_win.pin_memory(), k=lay.k.pin_memory(), v=lay.v.pin_memory(),
+                         ss=lay.seq_start, sl=lay.seq_len))
+    k_out = torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype).pin_memory()
+    v_out = torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype).pin_memory()
+    lengths = torch.zeros(units, dtype=torch.int32)
+    offsets = torch.zeros(units + 1, dtype=torch.int64)
+    kv_elems = host[0]["k"].numel()
+    arena = torch.empty(binding.refree_host_arena_size(params, total, kv_elems, cap), dtype=torch.uint8, device=dev)
+    d2h = 0
+
+    def one(h):
+        binding.refree_compress_layer_host(params, h["q"], h["k"], h["v"], h["ss"], h["sl"], total, k_out, v_out,
+                                           cap, lengths, offsets, None, None, arena)
+        return int(offsets[-1]) * 2 * row + lengths.numel() * 4 + offsets.numel() * 8 + 4
+
+    for h in host:
+        one(h)
+    reps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        for h in host:
+            d2h += one(h)
+    dt = time.perf_counter() - t0
+    per_layer = dt / (reps * n_lay)
+    h2d_layer = host[0]["q"].numel() * cfg.elem_bytes + 2 * kv_elems * cfg.elem_bytes + 8 * host[0]["sl"].numel()
+    return {"value": round(total / per_layer, 1), "unit": UNIT,
+            "h2d_bytes_per_step": int(h2d_layer * L), "d2h_bytes_per_step": int(d2h / (reps * n_lay) * L),
+            "ms_per_step": round(per_layer * L * 1e3, 3),
+            "how": f"refree_compress_layer_host on pinned host buffers, {n_lay} layers x {reps} sweeps, "
+                   f"wall clock (the call synchronises), scaled to {L} layers"}
+
+
+# --------------------------------------------------------- CPU oracle arm ----
+def oracle_sample(cfg, rank_mode, layer_idx, heads):
+    """Inputs of the oracle for `heads` KV heads of one layer of the workload."""
+    from oracle import refree_oracle as orc
+    from paper_2502_16886_b200 import workloads
+    lay = workloads.make_layer(cfg, layer_idx)
+    G = cfg.group
+    total = lay.total_tokens
+    p = orc.OracleParams(int(lay.seq_len.numel()), heads * G, heads, cfg.head_dim, window=cfg.window, sink=cfg.sink,
+                         rank_mode=rank_mode, dtype=0 if cfg.dtype == "fp32" else 1,
+                         k_strides=(0, cfg.head_dim, total * cfg.head_dim),
+                         v_strides=(0, cfg.head_dim, total * cfg.head_dim))
+    return p, lay.q_win[:, :heads * G].contiguous(), lay.k[:heads].contiguous(), lay.v[:heads].contiguous(), \
+        lay.seq_start, lay.seq_len
+
+
+def oracle_heads_for_budget(cfg, total, seconds=2.5):
+    """KV heads per sample so that one oracle call takes about `seconds` on this host."""
+    from oracle import refree_oracle as orc
+    macs_per_head = cfg.group * cfg.window * total * cfg.head_dim
+    rate = 1.2e9 * orc.num_threads()              # fp64 scalar multiply-adds per second, rough
+    return max(1, min(cfg.num_kv_heads, int(seconds * rate / macs_per_head)))
+
+
+def measure_cpu_baseline(cfg, rank_mode, total, args):
+    from oracle import build as obuild, refree_oracle as orc
+    obuild.build()
+    heads = oracle_heads_for_budget(cfg, total)
+    t_used, n_calls, layer = 0.0, 0, 0
+    while t_used < 10.0 and n_calls < 8:
+        inp = oracle_sample(cfg, rank_mode, layer % cfg.num_layers, heads)
+        t0 = time.perf_counter()
+        orc.compress_layer(*inp)
+        t_used += time.perf_counter() - t0
+        n_calls += 1
+        layer += 1
+    per_layer = t_used / n_calls * cfg.num_kv_heads / heads
+    return {"value": round(total / per_layer, 1), "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{n_calls} layer(s) of {cfg.name}, {heads} of {cfg.num_kv_heads} KV heads each, "
+                      f"scaled to a full layer; {t_used:.1f}s of CPU time"}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from oracle import build as obuild, refree_oracle as orc
+    from paper_2502_16886_b200 import workloads
+    obuild.build()
+    cfg = workloads.get_config(args.workload)
+    rank_mode = 1 if args.rank_mode == "score" else 0
+    seq_lens = workloads.sequence_lengths(cfg)
+    total = sum(seq_lens)
+    heads = oracle_heads_for_budget(cfg, total, seconds=2.0)
+    samples = [oracle_sample(cfg, rank_mode, l, heads) for l in range(min(2, cfg.num_layers))]
+    for i in range(args.warmup):
+        orc.compress_layer(*samples[i % len(samples)])
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        orc.compress_layer(*samples[i % len(samples)])
+    dt = (time.perf_counter() - t0) / args.steps
+    per_layer = dt * cfg.num_kv_heads / heads
+    value = round(total / per_layer, 1)
+    sample = (f"one step = one layer of {cfg.name}, {heads} of {cfg.num_kv_heads} KV heads, "
+              f"scaled to a full layer; host-resident inputs")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(per_layer * cfg.num_layers * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "layers": cfg.num_layers, "rank_mode": args.rank_mode, "window": cfg.window},
+            "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--rank-mode", choices=["position", "score"], default="position")
+    ap.add_argument("--layers", type=int, default=0, help="debugging: use fewer layers than the config")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 5
+        args.warmup = args.warmup if args.warmup is not None else 1
+        run_reference(args)
+    else:
+        args.steps = args.steps if args.steps is not None else 200
+        args.warmup = args.warmup if args.warmup is not None else 5
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

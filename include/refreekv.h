@@ -56,7 +56,8 @@ typedef enum {
     REFREE_ERR_CAPACITY = 4,
     REFREE_ERR_CUDA = 5,
     REFREE_ERR_TIMEOUT = 6,
-    REFREE_ERR_NONFINITE = 7
+    REFREE_ERR_NONFINITE = 7,
+    REFREE_ERR_STATIC_LIMIT = 8  /* problem too large for the built-in scratch of a *_static entry point */
 } refree_status;
 
 enum { REFREE_DEV_CAPACITY = 1, REFREE_DEV_TIMEOUT = 2, REFREE_DEV_NONFINITE = 4 };
@@ -156,6 +157,38 @@ refree_status refree_compress_layer_host(const refree_params *p, const void *q_w
                                          int32_t *lengths, int64_t *offsets,
                                          int32_t *kept_idx, float *scores,
                                          void *arena, size_t arena_bytes, void *stream);
+
+/* Selection without any device allocation (no counterpart in the paper; the
+ * arithmetic and the outputs are exactly those of refree_select_budget).
+ *
+ * Who needs it: code that may not create device memory at the point where it
+ * compresses a cache - a serving engine whose memory pool was carved up at
+ * start-up and has no slack left for a workspace, a plug-in running inside a
+ * host that forbids cudaMalloc after initialisation, a process whose allocator
+ * would synchronise the device in the middle of a latency-critical step.  Such
+ * callers own scores, lengths, offsets and kept_idx already (they are the
+ * stage's inputs and outputs) but cannot obtain the scratch that
+ * refree_select_budget takes as `workspace`.
+ *
+ * Here the scratch is a fixed array of REFREE_STATIC_SCRATCH_BYTES compiled into
+ * the library; every GPU that loads the library holds that many bytes until the
+ * process exits.  The call performs no cudaMalloc / cudaFree and uses no
+ * allocating routine.  A problem whose scratch need exceeds the array (roughly
+ * num_seqs * num_kv_heads > REFREE_STATIC_SCRATCH_BYTES / 24) is refused with
+ * REFREE_ERR_STATIC_LIMIT and nothing is launched.
+ *
+ * The first call on each device looks up the device address of the array
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * outside any stream capture.  All calls on a device share the one array: it
+ * keeps the previous call's contents, which is harmless because each call
+ * writes every record before reading it, but two calls whose kernels overlap
+ * on the GPU (different streams, no ordering between them) race on it. */
+#define REFREE_STATIC_SCRATCH_BYTES (256 * 1024)
+refree_status refree_select_budget_static(const refree_params *p, const float *scores,
+                                          const int32_t *seq_len, int64_t total_tokens,
+                                          int32_t *lengths, int64_t *offsets,
+                                          int32_t *kept_idx, int64_t capacity_rows,
+                                          int32_t *device_status, void *stream);
 
 /* Diagnostic with no counterpart in the paper: the number of CUDA kernels this
  * library has enqueued in this process so far (all entry points, all streams). */

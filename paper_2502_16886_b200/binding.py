@@ -15,7 +15,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "librefreekv.so")
 
 REFREE_OK = 0
-STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CAPACITY", "CUDA", "TIMEOUT", "NONFINITE"]
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CAPACITY", "CUDA", "TIMEOUT", "NONFINITE",
+                "STATIC_LIMIT"]
+STATIC_SCRATCH_BYTES = 256 * 1024
 DEV_CAPACITY, DEV_TIMEOUT, DEV_NONFINITE = 1, 2, 4
 RANK_POSITION, RANK_SCORE = 0, 1
 SCOPE_HEAD, SCOPE_LAYER = 0, 1
@@ -81,6 +83,7 @@ SIGNATURES = {
     "refree_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
     "refree_score": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
     "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
+    "refree_select_budget_static": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
@@ -162,6 +165,19 @@ def refree_select_budget(p: Params, scores, seq_len, total_tokens, lengths, offs
                                     _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_select_budget")
+    return rc
+
+
+def refree_select_budget_static(p: Params, scores, seq_len, total_tokens, lengths, offsets, kept_idx, capacity_rows,
+                                device_status=None, stream=None, check=True) -> int:
+    """Selection with the library's built-in scratch: takes no workspace and
+    allocates nothing (see the header for who needs this and for its limits)."""
+    c = p.c_struct()
+    rc = lib().refree_select_budget_static(ctypes.byref(c), _dp(scores), _dp(seq_len), total_tokens, _dp(lengths),
+                                           _dp(offsets), _dp(kept_idx), capacity_rows, _dp(device_status),
+                                           _stream(stream))
+    if check:
+        _check(rc, "refree_select_budget_static")
     return rc
 
 

@@ -111,6 +111,7 @@ const char *refree_status_string(refree_status s)
     case REFREE_ERR_CUDA: return "CUDA runtime error";
     case REFREE_ERR_TIMEOUT: return "a bounded on-device wait gave up";
     case REFREE_ERR_NONFINITE: return "non-finite score";
+    case REFREE_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
     }
     return "unknown status";
 }

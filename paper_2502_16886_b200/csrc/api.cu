@@ -1,6 +1,7 @@
 // C-ABI entry points: argument checks, workspace layout, launch sequences.
 #include <string.h>
 
+#include <algorithm>
 #include <atomic>
 
 #include "refree_internal.cuh"
@@ -20,8 +21,11 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     const int64_t rows = G * p.window;
     const int64_t tiles = total_tokens / kTile + p.num_seqs;
     size_t off = 0;
-    w.part_off = off;   w.part_bytes = align256((size_t)(tiles * p.num_kv_heads * rows) * sizeof(float2)); off += w.part_bytes;
-    w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows) * sizeof(float));                        off += w.lse_bytes;
+    // partials: per (tile, head, row) for the generic path, per (CTA + unit, padded row) for the tensor-core path
+    const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
+    const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
+    w.part_off = off;   w.part_bytes = align256((size_t)part_items * sizeof(float2));                      off += w.part_bytes;
+    w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
     w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
     w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
     w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
@@ -73,7 +77,7 @@ static cudaError_t run_score(const refree_params &p, const void *q_win, const vo
                              float *scores, char *ws, const Workspace &lay, int32_t *dev_status,
                              cudaStream_t st)
 {
-    if (score_tc_supported(p))
+    if (score_tc_supported(p) && !(reinterpret_cast<uintptr_t>(q_win) & 15))
         return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
     return launch_score_generic(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
 }

@@ -1,10 +1,758 @@
-// Tensor-core scoring path (placeholder until the tcgen05 kernels land).
+// Tensor-core scoring path (steps S1-S3) for bf16 caches with head_dim 128.
+//
+// The window logits S = Q K^T are the one dense contraction of the pass; they run
+// on tcgen05.mma with the accumulator in tensor memory, operands staged in shared
+// memory by TMA (128-byte swizzle).  A row's softmax normaliser needs all of the
+// row, and the column sums need every row's normaliser, so the logits are formed
+// twice (storing them would cost more HBM traffic than K itself):
+//
+//   pass 1  D[row, position] = Q_blk K_tile^T : one thread per query row sums
+//           2^(y - c) over the positions it may see (no cross-thread traffic);
+//           partial (c, Z) per (CTA, unit) go to the workspace
+//   combine L[row] = log2 sum_i 2^(y_i) from the partials
+//   pass 2  D[position, row] = K_tile Q^T : one thread per position sums
+//           2^(y - L[row]) over the rows that see it -> a'[i]  (Eq. 2)
+//
+// Both passes use the same shared-memory images of Q and K (K-major, so either
+// can be the A or the B operand); only the roles swap, which puts each pass's
+// reduction inside a thread.  Persistent CTAs (one per SM) take contiguous ranges
+// of (unit, tile) items; warp 8 issues TMA, warp 9 issues MMA, warps 0-7 are the
+// epilogue (two warpgroups, each on one half of a 256-column accumulator, two
+// accumulators in flight).  Every wait is bounded: on a timeout the CTA records
+// REFREE_DEV_TIMEOUT, stops issuing work, and falls through to the common exit
+// where tensor memory is released.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
 #include "refree_internal.cuh"
+
 namespace refree {
-bool score_tc_supported(const refree_params &) { return false; }
-cudaError_t launch_score_tc(const refree_params &, const void *, const void *, const int32_t *, const int32_t *,
-                            int64_t, float *, char *, const Workspace &, int32_t *, cudaStream_t)
+namespace {
+
+constexpr int kEpiWarps = 8;
+constexpr int kThreadsTc = (kEpiWarps + 2) * 32;
+constexpr int kD = 128;
+constexpr int kHalfBytes = kTile * 128;          // one 64-column half of a 128-row tile: 16 KB
+constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KB
+constexpr int kMaxRowsTc = 512;
+constexpr int kMaxCtas = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kZLimit = 1.2676506e30f;         // 2^100: a tile sum above this is redone with a fresh reference
+
+// ------------------------------------------------------------------ PTX ------
+__device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint64_t *bar, uint32_t count)
 {
-    return cudaErrorNotSupported;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ inline void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ inline void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline bool mbar_try(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when it gives up.
+__device__ inline bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if (it > 64) {
+            if (*abort_flag) return false;
+            __nanosleep(it > 4096 ? 256 : 32);
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ inline void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ inline void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ inline void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ inline void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ inline void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+__device__ inline void tmem_alloc(uint32_t *dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival once every MMA issued so far by this thread has completed.
+__device__ inline void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ inline void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ inline float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B
+// apart, groups of 8 rows 1024 B apart (the layout TMA writes with SWIZZLE_128B).
+__device__ inline uint64_t make_desc(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset: 8 rows * 128 B
+    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ inline uint32_t make_idesc(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ---------------------------------------------------------------- shapes -----
+struct TcShape {
+    int R;        // query rows per unit: G * window
+    int Rpad;     // rows of the shared-memory Q image (multiple of 128)
+    int rblocks;  // 128-row blocks (pass 1 A operands)
+    int jobs1;    // pass-1 accumulators per tile (two row blocks each)
+    int nb;       // pass-2 accumulators per tile
+    int ncol;     // pass-2 columns (rows of Q) per accumulator: R / nb
+    int stages;   // K tile ring depth
+    int rank4;    // K tensor map has a sequence axis
+};
+
+struct TcSmemTail {
+    uint64_t k_full[4], k_empty[4], q_full, q_empty, acc_full[2], acc_empty[2], epi_bar;
+    uint32_t tmem_base;
+    int abort_flag;
+    alignas(16) float stage[2][2][kTile];     // pass 2: per item parity, per warpgroup partial column sums
+    alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
+    SeqTables seq;
+};
+
+struct ItemTc {
+    int u, s, g, n, tile_start, tok0, pack;
+};
+
+__device__ inline ItemTc decode_item_tc(const SeqTables &t, const int32_t *seq_start, const int32_t *seq_len,
+                                        int B, int Hkv, int item)
+{
+    // items are ordered (sequence, head, tile): a CTA's consecutive items mostly share a unit
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((int64_t)t.tiles[mid] * Hkv <= item) lo = mid; else hi = mid;
+    }
+    ItemTc it;
+    it.s = lo;
+    const int ts = t.tiles[lo + 1] - t.tiles[lo];
+    const int rem = item - t.tiles[lo] * Hkv;
+    it.g = rem / ts;
+    it.tile_start = (rem % ts) * kTile;
+    it.u = lo * Hkv + it.g;
+    it.n = seq_len[lo];
+    it.tok0 = seq_start[lo];
+    it.pack = t.pack[lo];
+    return it;
+}
+
+// first item of CTA c when `items` are split evenly over `ctas`
+__device__ __host__ inline int range_begin(int c, int items, int ctas) { return (int)((int64_t)c * items / ctas); }
+
+struct TcArgs {
+    refree_params p;
+    TcShape sh;
+    const int32_t *seq_start, *seq_len;
+    float2 *part;        // [ctas + units][Rpad]
+    float *lse;          // [units][Rpad]
+    float *scores;
+    int64_t total_tokens;
+    int32_t *dev_status;
+};
+
+// Barrier among the epilogue warps, built on an mbarrier so that it is bounded like
+// every other wait of the kernel (one arrival per warp).
+__device__ inline bool epi_sync(TcSmemTail &tl, uint32_t &phase)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(&tl.epi_bar);
+    const bool ok = mbar_wait(&tl.epi_bar, phase, &tl.abort_flag);
+    phase ^= 1;
+    return ok;
+}
+
+// --------------------------------------------------------- producer / MMA -----
+template <int PASS>
+__device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, const CUtensorMap *mapk,
+                                     unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
+                                     int item0, int item1)
+{
+    const TcShape &sh = a.sh;
+    const int G = a.p.num_q_heads / a.p.num_kv_heads;
+    int cur_u = -1, stage = 0;
+    uint32_t kphase = 0, qphase = 0;
+    bool ok = true;
+    for (int item = item0; item < item1 && ok; ++item) {
+        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+        if (it.u != cur_u) {
+            ok = mbar_wait(&tl.q_empty, qphase ^ 1, &tl.abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(&tl.q_full, (uint32_t)sh.Rpad * 256u);
+            const int row0 = (it.s * a.p.num_q_heads + it.g * G) * a.p.window;
+            for (int h = 0; h < 2; ++h)
+                for (int rb = 0; rb < sh.rblocks; ++rb)
+                    tma_load_2d(smem_q + (size_t)h * sh.Rpad * 128 + (size_t)rb * kHalfBytes, mapq, &tl.q_full,
+                                h * 64, row0 + rb * kTile);
+            qphase ^= 1;
+            cur_u = it.u;
+        }
+        ok = mbar_wait(&tl.k_empty[stage], kphase ^ 1, &tl.abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(&tl.k_full[stage], (uint32_t)kTileBytes);
+        unsigned char *dst = smem_k + (size_t)stage * kTileBytes;
+        for (int h = 0; h < 2; ++h) {
+            if (sh.rank4)
+                tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s);
+            else
+                tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g);
+        }
+        if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
+    }
+    // Before leaving, let every copy this thread started land (bounded): the ring's
+    // full barriers complete only when their bytes have arrived.
+    if (!ok) {
+        for (int s2 = 0; s2 < sh.stages; ++s2)
+            for (uint32_t itw = 0; itw < 4096; ++itw) {
+                if (mbar_try(&tl.k_full[s2], 0) || mbar_try(&tl.k_full[s2], 1)) break;
+                __nanosleep(64);
+            }
+    }
+}
+
+template <int PASS>
+__device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
+                                uint32_t tmem_base, int item0, int item1)
+{
+    const TcShape &sh = a.sh;
+    const uint32_t q_addr = smem_u32(smem_q), k_addr = smem_u32(smem_k);
+    const uint32_t idesc1 = make_idesc(kTile), idesc2 = make_idesc(sh.ncol);
+    int cur_u = -1, stage = 0, buf = 0;
+    uint32_t kphase = 0, qphase = 0, aphase[2] = {0, 0};
+    bool ok = true;
+    int prev_u = -1;
+    for (int item = item0; item < item1 && ok; ++item) {
+        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+        if (it.u != cur_u) {
+            if (prev_u >= 0) umma_commit(&tl.q_empty);     // every MMA on the previous unit's Q has been issued
+            ok = mbar_wait(&tl.q_full, qphase, &tl.abort_flag);
+            if (!ok) break;
+            qphase ^= 1;
+            cur_u = it.u;
+            prev_u = it.u;
+        }
+        ok = mbar_wait(&tl.k_full[stage], kphase, &tl.abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t kt = k_addr + (uint32_t)stage * kTileBytes;
+        const int jobs = PASS == 1 ? sh.jobs1 : sh.nb;
+        for (int job = 0; job < jobs && ok; ++job) {
+            ok = mbar_wait(&tl.acc_empty[buf], aphase[buf] ^ 1, &tl.abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d0 = tmem_base + (uint32_t)buf * 256u;
+            if (PASS == 1) {
+                for (int half_acc = 0; half_acc < 2; ++half_acc) {
+                    const int rb = 2 * job + half_acc;
+                    if (rb >= sh.rblocks) break;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t h = kk >> 2, ko = (kk & 3) * 32;
+                        umma_bf16(d0 + half_acc * 128,
+                                  make_desc(q_addr + h * sh.Rpad * 128 + rb * kHalfBytes + ko),
+                                  make_desc(kt + h * kHalfBytes + ko), idesc1, kk > 0);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t h = kk >> 2, ko = (kk & 3) * 32;
+                    umma_bf16(d0, make_desc(kt + h * kHalfBytes + ko),
+                              make_desc(q_addr + h * sh.Rpad * 128 + job * sh.ncol * 128 + ko), idesc2, kk > 0);
+                }
+            }
+            umma_commit(&tl.acc_full[buf]);
+            aphase[buf] ^= 1;
+            buf ^= 1;
+        }
+        umma_commit(&tl.k_empty[stage]);
+        if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
+    }
+}
+
+// ------------------------------------------------------------- epilogues -----
+// Pass 1: thread = query row.  Sum of 2^(y - c) over the positions the row sees.
+template <bool MASKED>
+__device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, int limit)
+{
+    float z0 = 0.f, z1 = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+            float e0 = ex2(fmaf(v[i], scale, -cref));
+            float e1 = ex2(fmaf(v[i + 1], scale, -cref));
+            if (MASKED) {
+                e0 = (c * 32 + i < limit) ? e0 : 0.f;
+                e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
+            }
+            z0 += e0;
+            z1 += e1;
+        }
+    }
+    return z0 + z1;
+}
+__device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
+{
+    float m = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (c * 32 + i < limit) m = fmaxf(m, v[i] * scale);
+    }
+    return m;
+}
+
+__device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1)
+{
+    const TcShape &sh = a.sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wg = warp >> 2, lane_base = (warp & 3) * 32;
+    const float scale = kLog2e * rsqrtf((float)kD);
+    const int w = a.p.window;
+    int cur_u = -1, buf = 0;
+    uint32_t aphase[2] = {0, 0};
+    // per job slot (row block 2*job + wg): running reference and sum of this thread's row
+    float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
+    bool ok = true;
+    auto flush = [&](int u) {
+        for (int job = 0; job < sh.jobs1; ++job) {
+            const int rb = 2 * job + wg;
+            const int row = rb * kTile + lane_base + lane;
+            if (rb < sh.rblocks && row < sh.R)
+                a.part[(int64_t)(blockIdx.x + u) * sh.Rpad + row] = make_float2(cref[job], zsum[job]);
+            cref[job] = -INFINITY;
+            zsum[job] = 0.f;
+        }
+    };
+    for (int item = item0; item < item1 && ok; ++item) {
+        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+        if (it.u != cur_u) {
+            if (cur_u >= 0) flush(cur_u);
+            cur_u = it.u;
+        }
+        for (int job = 0; job < sh.jobs1 && ok; ++job) {
+            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int rb = 2 * job + wg;
+            if (rb < sh.rblocks) {
+                const int row = rb * kTile + lane_base + lane;
+                const int pos = it.n - w + (row % w);               // position of this row's query
+                int limit = pos - it.tile_start + 1;                // visible positions of the tile: [0, limit)
+                limit = (row < sh.R) ? max(0, min(kTile, limit)) : 0;
+                const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)wg * 128u + ((uint32_t)lane_base << 16);
+                const bool full = __all_sync(0xffffffffu, limit == kTile);
+                bool need_max = (cref[job] == -INFINITY) && limit > 0;
+                float zt = 0.f;
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    if (__any_sync(0xffffffffu, need_max)) {
+                        const float m = row_max_tile(taddr, scale, limit);
+                        if (need_max && m > cref[job]) {
+                            zsum[job] = (cref[job] == -INFINITY) ? 0.f : zsum[job] * ex2(cref[job] - m);
+                            cref[job] = m;
+                        }
+                    }
+                    zt = full ? row_sum_tile<false>(taddr, scale, cref[job], limit)
+                              : row_sum_tile<true>(taddr, scale, cref[job], limit);
+                    need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
+                    if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
+                }
+                if (limit > 0) zsum[job] += zt;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
+            aphase[buf] ^= 1;
+            buf ^= 1;
+        }
+    }
+    if (cur_u >= 0 && ok) flush(cur_u);
+}
+
+// Pass 2: thread = position.  Sum over the rows that see it of 2^(y - L[row]).
+template <bool MASKED, int W>
+__device__ inline float col_sum_chunk(uint32_t taddr, float scale, const float *lse, int r0, int w, int pos_gap)
+{
+    // pos_gap = i - (n - w): row r sees position i iff (r mod w) >= pos_gap
+    float v[W];
+    if (W == 32) tmem_ld32(taddr, *reinterpret_cast<float (*)[32]>(v));
+    else tmem_ld16(taddr, *reinterpret_cast<float (*)[16]>(v));
+    float s0 = 0.f, s1 = 0.f;
+    int rloc = MASKED ? r0 % w : 0;
+#pragma unroll
+    for (int i = 0; i < W; i += 4) {
+        const float4 L = *reinterpret_cast<const float4 *>(lse + r0 + i);
+        float e[4];
+        e[0] = ex2(fmaf(v[i], scale, -L.x));
+        e[1] = ex2(fmaf(v[i + 1], scale, -L.y));
+        e[2] = ex2(fmaf(v[i + 2], scale, -L.z));
+        e[3] = ex2(fmaf(v[i + 3], scale, -L.w));
+        if (MASKED) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (rloc < pos_gap) e[j] = 0.f;
+                if (++rloc == w) rloc = 0;
+            }
+        }
+        s0 += e[0] + e[2];
+        s1 += e[1] + e[3];
+    }
+    return s0 + s1;
+}
+
+__device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1)
+{
+    const TcShape &sh = a.sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wg = warp >> 2, lane_base = (warp & 3) * 32;
+    const int tid = threadIdx.x;                                   // 0..255
+    const float scale = kLog2e * rsqrtf((float)kD);
+    const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads;
+    const int ncol_wg = sh.ncol / 2;                               // columns per warpgroup (multiple of 16)
+    int cur_u = -1, buf = 0, par = 0;
+    uint32_t aphase[2] = {0, 0}, ephase = 0;
+    bool ok = true;
+    for (int item = item0; item < item1 && ok; ++item) {
+        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+        if (it.u != cur_u) {
+            if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
+            for (int r = tid; r < sh.R; r += kEpiWarps * 32) tl.lse[r] = a.lse[(int64_t)it.u * sh.Rpad + r];
+            if (!(ok = epi_sync(tl, ephase))) break;
+            cur_u = it.u;
+        }
+        const int pos_in_tile = lane_base + lane;
+        const int i = it.tile_start + pos_in_tile;
+        const int pos_gap = i - (it.n - w);
+        // tile wholly before the window and wholly inside the sequence: every row sees every position
+        const bool full = it.tile_start + kTile <= it.n - w + 1;
+        float acc = 0.f;
+        for (int job = 0; job < sh.nb && ok; ++job) {
+            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)(wg * ncol_wg) + ((uint32_t)lane_base << 16);
+            const int rbase = job * sh.ncol + wg * ncol_wg;
+            int c = 0;
+            for (; c + 32 <= ncol_wg; c += 32)
+                acc += full ? col_sum_chunk<false, 32>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap)
+                            : col_sum_chunk<true, 32>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap);
+            if (c < ncol_wg)
+                acc += full ? col_sum_chunk<false, 16>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap)
+                            : col_sum_chunk<true, 16>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
+            aphase[buf] ^= 1;
+            buf ^= 1;
+        }
+        if (!ok) break;
+        tl.stage[par][wg][pos_in_tile] = acc;
+        if (!(ok = epi_sync(tl, ephase))) break;
+        if (wg == 0 && i < it.n) {
+            const float tot = tl.stage[par][0][pos_in_tile] + tl.stage[par][1][pos_in_tile];
+            const int cnt = min(min(w, it.n), it.n - i);
+            const float sc = tot / (float)cnt / (float)G;
+            if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
+            a.scores[(int64_t)it.g * a.total_tokens + it.pack + i] = sc;
+        }
+        par ^= 1;     // the other staging buffer is free: its readers passed this item's barrier
+    }
+}
+
+// ---------------------------------------------------------------- kernels ----
+template <int PASS>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant__ CUtensorMap mapk, TcArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const TcShape &sh = a.sh;
+    unsigned char *smem_q = smem;
+    unsigned char *smem_k = smem + (size_t)sh.Rpad * 256;
+    TcSmemTail &tl = *reinterpret_cast<TcSmemTail *>(smem_k + (size_t)sh.stages * kTileBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 4; ++s) { mbar_init(&tl.k_full[s], 1); mbar_init(&tl.k_empty[s], 1); }
+        mbar_init(&tl.q_full, 1);
+        mbar_init(&tl.q_empty, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps); }
+        mbar_init(&tl.epi_bar, kEpiWarps);
+        tl.abort_flag = 0;
+        fence_barrier_init();
+    }
+    build_seq_tables(tl.seq, a.seq_len, a.p.num_seqs);       // ends with __syncthreads()
+    if (warp == kEpiWarps + 1) tmem_alloc(&tl.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tl.tmem_base;
+
+    const int items = tl.seq.tiles[a.p.num_seqs] * a.p.num_kv_heads;
+    const int item0 = range_begin(blockIdx.x, items, gridDim.x), item1 = range_begin(blockIdx.x + 1, items, gridDim.x);
+
+    if (warp < kEpiWarps) {
+        if (PASS == 1) epilogue_pass1(a, tl, tmem_base, item0, item1);
+        else epilogue_pass2(a, tl, tmem_base, item0, item1);
+    } else if (warp == kEpiWarps) {
+        if (lane == 0) producer_loop<PASS>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1);
+    } else {
+        if (lane == 0) mma_loop<PASS>(a, smem_q, smem_k, tl, tmem_base, item0, item1);
+    }
+    __syncwarp();
+    // Common exit.  In the normal case the epilogue has consumed every accumulator,
+    // which implies every MMA and every copy has completed.
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (threadIdx.x == 0 && tl.abort_flag && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_TIMEOUT);
+    if (warp == kEpiWarps + 1) tmem_dealloc(tmem_base, 512);
+}
+
+// L[u][row] = log2 sum over the row's visible positions of 2^y, from the per-(CTA, unit) partials.
+__global__ void score_tc_combine(TcArgs a, int ctas)
+{
+    __shared__ SeqTables seq;
+    const TcShape &sh = a.sh;
+    const int B = a.p.num_seqs, Hkv = a.p.num_kv_heads;
+    build_seq_tables(seq, a.seq_len, B);
+    const int items = seq.tiles[B] * Hkv;
+    const int64_t total = (int64_t)B * Hkv * sh.R;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int row = (int)(e % sh.R), u = (int)(e / sh.R);
+        const int s = u / Hkv, g = u % Hkv;
+        const int ts = seq.tiles[s + 1] - seq.tiles[s];
+        float L = INFINITY;                                   // a row that sees nothing contributes 2^(-inf) = 0
+        if (ts > 0) {
+            const int ib = seq.tiles[s] * Hkv + g * ts, ie = ib + ts;      // the unit's items
+            // CTAs whose ranges meet [ib, ie)
+            int c0 = (int)(((int64_t)ib * ctas) / items);
+            while (c0 > 0 && range_begin(c0, items, ctas) > ib) --c0;
+            while (c0 + 1 < ctas && range_begin(c0 + 1, items, ctas) <= ib) ++c0;
+            float m = -INFINITY;
+            // a CTA took part in the unit iff its (non-empty) range meets [ib, ie)
+            auto meets = [&](int c) {
+                const int b0 = range_begin(c, items, ctas), b1 = range_begin(c + 1, items, ctas);
+                return b1 > b0 && b1 > ib && b0 < ie;
+            };
+            for (int c = c0; c < ctas && range_begin(c, items, ctas) < ie; ++c)
+                if (meets(c)) m = fmaxf(m, a.part[(int64_t)(c + u) * sh.Rpad + row].x);
+            float z = 0.f;
+            for (int c = c0; c < ctas && range_begin(c, items, ctas) < ie; ++c) {
+                if (!meets(c)) continue;
+                const float2 pr = a.part[(int64_t)(c + u) * sh.Rpad + row];
+                if (pr.y > 0.f) z += pr.y * exp2f(pr.x - m);
+            }
+            if (z > 0.f) L = m + log2f(z);
+        }
+        a.lse[(int64_t)u * sh.Rpad + row] = L;
+    }
+}
+
+// ------------------------------------------------------------------ host -----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool shape_for(const refree_params &p, TcShape &sh)
+{
+    if (p.dtype != REFREE_DTYPE_BF16 || p.head_dim != kD) return false;
+    const int G = p.num_q_heads / p.num_kv_heads;
+    const int64_t R = (int64_t)G * p.window;
+    if (R < 32 || R > kMaxRowsTc) return false;
+    sh.R = (int)R;
+    sh.nb = (sh.R + 255) / 256;
+    if (sh.R % (32 * sh.nb) != 0) return false;           // each warpgroup takes ncol/2 columns in chunks of 16
+    sh.ncol = sh.R / sh.nb;
+    sh.rblocks = (sh.R + kTile - 1) / kTile;
+    sh.Rpad = sh.rblocks * kTile;
+    sh.jobs1 = (sh.rblocks + 1) / 2;
+    sh.stages = sh.Rpad <= 256 ? 4 : 2;
+    sh.rank4 = p.k_stride_seq != 0;
+    return true;
+}
+
+size_t smem_bytes(const TcShape &sh)
+{
+    return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + sizeof(TcSmemTail);
+}
+
+}  // namespace
+
+bool score_tc_supported(const refree_params &p)
+{
+    TcShape sh;
+    if (!shape_for(p, sh)) return false;
+    if (p.kv_tokens <= 0 || p.kv_tokens > 0x7fffffffLL) return false;
+    return encode_fn() != nullptr;
+}
+
+cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
+                            const int32_t *seq_start, const int32_t *seq_len,
+                            int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
+                            int32_t *dev_status, cudaStream_t st)
+{
+    TcShape sh;
+    if (!shape_for(p, sh)) return cudaErrorInvalidValue;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap mapq, mapk;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_seqs * p.num_q_heads * p.window};
+        const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+        const cuuint32_t box[2] = {64, kTile}, estr[2] = {1, 1};
+        if (enc(&mapq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(q_win), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)p.kv_tokens, (cuuint64_t)p.num_kv_heads, (cuuint64_t)p.num_seqs};
+        const cuuint64_t strides[3] = {(cuuint64_t)p.k_stride_tok * 2, (cuuint64_t)p.k_stride_head * 2,
+                                       (cuuint64_t)p.k_stride_seq * 2};
+        const cuuint32_t box[4] = {64, kTile, 1, 1}, estr[4] = {1, 1, 1, 1};
+        if (enc(&mapk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, sh.rank4 ? 4 : 3, const_cast<void *>(k), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    static int sm_count[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = std::min(n, kMaxCtas);
+    }
+    const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
+    const int ctas = (int)std::max<int64_t>(1, std::min<int64_t>(sm_count[dev], max_items));
+    TcArgs a;
+    a.p = p;
+    a.sh = sh;
+    a.seq_start = seq_start;
+    a.seq_len = seq_len;
+    a.part = reinterpret_cast<float2 *>(ws + lay.part_off);
+    a.lse = reinterpret_cast<float *>(ws + lay.lse_off);
+    a.scores = scores;
+    a.total_tokens = total_tokens;
+    a.dev_status = dev_status;
+    const size_t smem = smem_bytes(sh);
+    if (smem > 232448) return cudaErrorInvalidValue;
+    score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
+    const int64_t rows = (int64_t)p.num_seqs * p.num_kv_heads * sh.R;
+    score_tc_combine<<<(int)std::min<int64_t>((rows + 255) / 256, 1024), 256, 0, st>>>(a, ctas);
+    score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
+    count_launches(3);
+    return cudaGetLastError();
+}
+
 }  // namespace refree

@@ -179,8 +179,8 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
     if (st != REFREE_OK) return st;
     if ((reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
         return REFREE_ERR_UNSUPPORTED;
-    return from_cuda(launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept_idx, false, k_out, v_out,
-                                    capacity_rows, device_status, (cudaStream_t)stream));
+    return from_cuda(launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept_idx, false, nullptr, k_out,
+                                    v_out, capacity_rows, device_status, (cudaStream_t)stream));
 }
 
 refree_status refree_compress_layer(const refree_params *p, const void *q_win,
@@ -215,10 +215,13 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
     if (total_tokens > 0 && (!p->force_full || scores))
         e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs);
     if (e != cudaSuccess) return REFREE_ERR_CUDA;
-    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs);
+    // with two-range kept sets and no index list wanted, the compaction kernel forms the offsets itself
+    const bool lean = ranges && !kept;
+    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs,
+                      !lean);
     if (e != cudaSuccess) return REFREE_ERR_CUDA;
-    e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, k_out, v_out, capacity_rows,
-                       device_status, cs);
+    e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, lean ? offsets : nullptr, k_out,
+                       v_out, capacity_rows, device_status, cs);
     return from_cuda(e);
 }
 

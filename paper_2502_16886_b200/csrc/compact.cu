@@ -27,9 +27,10 @@ __device__ inline void st_stream(int4 *p, const int4 &v)
 __global__ void __launch_bounds__(kThreads)
 compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq_start,
                const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
-               const int32_t *kept_idx, int position_ranges, char *k_out, char *v_out,
+               const int32_t *kept_idx, int position_ranges, int64_t *offsets_out, char *k_out, char *v_out,
                int64_t capacity_rows, int32_t *dev_status)
 {
+    __shared__ long long s_part[kThreads / 32];
     const int Hkv = p.num_kv_heads;
     const int u = blockIdx.y, s = u / Hkv, g = u % Hkv;
     const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
@@ -38,7 +39,23 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
     const int vshift = 31 - __clz(vec_per_row);
     const int n = max(seq_len[s], 0);
     const int b = lengths[u];
-    const int64_t off = offsets[u];
+    int64_t off;
+    if (offsets_out) {
+        // fused pass: the running sum of the budgets is formed here instead of in a launch of its own
+        long long part = 0;
+        for (int t = threadIdx.x; t < u; t += kThreads) part += lengths[t];
+        for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = part;
+        __syncthreads();
+        off = 0;
+        for (int wv = 0; wv < kThreads / 32; ++wv) off += s_part[wv];
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            offsets_out[u] = off;
+            if (u == (int)gridDim.y - 1) offsets_out[u + 1] = off + b;
+        }
+    } else {
+        off = offsets[u];
+    }
     if (b < 0 || b > n || off < 0 || off + b > capacity_rows) {
         if (threadIdx.x == 0 && blockIdx.x == 0 && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
         return;
@@ -80,13 +97,13 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            const int32_t *seq_start, const int32_t *seq_len,
                            const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
-                           bool position_ranges, void *k_out, void *v_out, int64_t capacity_rows,
-                           int32_t *dev_status, cudaStream_t st)
+                           bool position_ranges, int64_t *offsets_out, void *k_out, void *v_out,
+                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st)
 {
     const int U = p.num_seqs * p.num_kv_heads;
     const int gx = max(1, (148 * 8) / U);
     compact_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
-                                                     lengths, offsets, kept_idx, position_ranges ? 1 : 0,
+                                                     lengths, offsets, kept_idx, position_ranges ? 1 : 0, offsets_out,
                                                      (char *)k_out, (char *)v_out, capacity_rows, dev_status);
     count_launches(1);
     return cudaGetLastError();

@@ -102,12 +102,12 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
 cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
                           int64_t total_tokens, int32_t *lengths, int64_t *offsets,
                           int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,
-                          int32_t *dev_status, cudaStream_t st);
+                          int32_t *dev_status, cudaStream_t st, bool emit = true);
 
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            const int32_t *seq_start, const int32_t *seq_len,
                            const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
-                           bool position_ranges, void *k_out, void *v_out, int64_t capacity_rows,
-                           int32_t *dev_status, cudaStream_t st);
+                           bool position_ranges, int64_t *offsets_out, void *k_out, void *v_out,
+                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st);
 
 }  // namespace refree

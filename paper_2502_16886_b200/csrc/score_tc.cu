@@ -9,9 +9,9 @@
 //   pass 1  D[row, position] = Q_blk K_tile^T : one thread per query row sums
 //           2^(y - c) over the positions it may see (no cross-thread traffic);
 //           partial (c, Z) per (CTA, unit) go to the workspace
-//   combine L[row] = log2 sum_i 2^(y_i) from the partials
-//   pass 2  D[position, row] = K_tile Q^T : one thread per position sums
-//           2^(y - L[row]) over the rows that see it -> a'[i]  (Eq. 2)
+//   pass 2  on entering a unit, L[row] = log2 sum_i 2^(y_i) is merged from those
+//           partials; then D[position, row] = K_tile Q^T : one thread per position
+//           sums 2^(y - L[row]) over the rows that see it -> a'[i]  (Eq. 2)
 //
 // Both passes use the same shared-memory images of Q and K (K-major, so either
 // can be the A or the B operand); only the roles swap, which puts each pass's
@@ -120,32 +120,29 @@ __device__ inline void umma_commit(uint64_t *bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ inline void tmem_ld32(uint32_t taddr, float (&v)[32])
+// Tensor-memory loads are split into issue and wait so that the next chunk can be
+// in flight while the current one is consumed.  The wait names the destination
+// registers as in/out operands: the compiler must not read them before it.
+#define RF_OUT16(r, o) "=r"(r[o+0]), "=r"(r[o+1]), "=r"(r[o+2]), "=r"(r[o+3]), "=r"(r[o+4]), "=r"(r[o+5]), "=r"(r[o+6]), "=r"(r[o+7]), \
+                       "=r"(r[o+8]), "=r"(r[o+9]), "=r"(r[o+10]), "=r"(r[o+11]), "=r"(r[o+12]), "=r"(r[o+13]), "=r"(r[o+14]), "=r"(r[o+15])
+#define RF_IO16(r, o) "+r"(r[o+0]), "+r"(r[o+1]), "+r"(r[o+2]), "+r"(r[o+3]), "+r"(r[o+4]), "+r"(r[o+5]), "+r"(r[o+6]), "+r"(r[o+7]), \
+                      "+r"(r[o+8]), "+r"(r[o+9]), "+r"(r[o+10]), "+r"(r[o+11]), "+r"(r[o+12]), "+r"(r[o+13]), "+r"(r[o+14]), "+r"(r[o+15])
+__device__ inline void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
                  "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                 : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                 : RF_OUT16(r, 0), RF_OUT16(r, 16) : "r"(taddr) : "memory");
 }
-__device__ inline void tmem_ld16(uint32_t taddr, float (&v)[16])
+__device__ inline void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[16];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-                 : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+                 : RF_OUT16(r, 0) : "r"(taddr) : "memory");
+}
+__device__ inline void tmem_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : RF_IO16(r, 0), RF_IO16(r, 16) :: "memory");
 }
 __device__ inline float ex2(float x)
 {
@@ -227,7 +224,6 @@ struct TcArgs {
     TcShape sh;
     const int32_t *seq_start, *seq_len;
     float2 *part;        // [ctas + units][Rpad]
-    float *lse;          // [units][Rpad]
     float *scores;
     int64_t total_tokens;
     int32_t *dev_status;
@@ -358,14 +354,19 @@ template <bool MASKED>
 __device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, int limit)
 {
     float z0 = 0.f, z1 = 0.f;
+    const float nc = -cref;
+    uint32_t ra[32], rb[32];
+    tmem_ld32_issue(taddr, ra);
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(taddr + c * 32, v);
+        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+        tmem_ld_wait(cur);
+        if (c + 1 < 4) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-            float e0 = ex2(fmaf(v[i], scale, -cref));
-            float e1 = ex2(fmaf(v[i + 1], scale, -cref));
+            float e0 = ex2(fmaf(__uint_as_float(cur[i]), scale, nc));
+            float e1 = ex2(fmaf(__uint_as_float(cur[i + 1]), scale, nc));
             if (MASKED) {
                 e0 = (c * 32 + i < limit) ? e0 : 0.f;
                 e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
@@ -379,13 +380,17 @@ __device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, in
 __device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
 {
     float m = -INFINITY;
+    uint32_t ra[32], rb[32];
+    tmem_ld32_issue(taddr, ra);
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(taddr + c * 32, v);
+        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+        tmem_ld_wait(cur);
+        if (c + 1 < 4) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-            if (c * 32 + i < limit) m = fmaxf(m, v[i] * scale);
+            if (c * 32 + i < limit) m = fmaxf(m, __uint_as_float(cur[i]) * scale);
     }
     return m;
 }
@@ -458,53 +463,93 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
 }
 
 // Pass 2: thread = position.  Sum over the rows that see it of 2^(y - L[row]).
-template <bool MASKED, int W>
-__device__ inline float col_sum_chunk(uint32_t taddr, float scale, const float *lse, int r0, int w, int pos_gap)
+// One accumulator's share of a warpgroup: ncol_wg columns (a multiple of 16, at most
+// 128) taken in chunks of 32 (the last may be 16), next chunk in flight.
+template <bool MASKED>
+__device__ inline float col_sum_job(uint32_t taddr, float scale, const float *lse, int rbase, int ncol_wg,
+                                    int w, int pos_gap)
 {
     // pos_gap = i - (n - w): row r sees position i iff (r mod w) >= pos_gap
-    float v[W];
-    if (W == 32) tmem_ld32(taddr, *reinterpret_cast<float (*)[32]>(v));
-    else tmem_ld16(taddr, *reinterpret_cast<float (*)[16]>(v));
+    uint32_t ra[32] = {}, rb[32] = {};
     float s0 = 0.f, s1 = 0.f;
-    int rloc = MASKED ? r0 % w : 0;
+    if (ncol_wg >= 32) tmem_ld32_issue(taddr, ra); else tmem_ld16_issue(taddr, ra);
 #pragma unroll
-    for (int i = 0; i < W; i += 4) {
-        const float4 L = *reinterpret_cast<const float4 *>(lse + r0 + i);
-        float e[4];
-        e[0] = ex2(fmaf(v[i], scale, -L.x));
-        e[1] = ex2(fmaf(v[i + 1], scale, -L.y));
-        e[2] = ex2(fmaf(v[i + 2], scale, -L.z));
-        e[3] = ex2(fmaf(v[i + 3], scale, -L.w));
-        if (MASKED) {
+    for (int c = 0; c < 4; ++c) {
+        if (c * 32 < ncol_wg) {
+            uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+            uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+            tmem_ld_wait(cur);
+            if (c + 1 < 4 && (c + 1) * 32 < ncol_wg) {
+                if (ncol_wg - (c + 1) * 32 >= 32) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
+                else tmem_ld16_issue(taddr + (c + 1) * 32, nxt);
+            }
+            const int r0 = rbase + c * 32;
+            const int width = min(32, ncol_wg - c * 32);
+            int rloc = MASKED ? r0 % w : 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (rloc < pos_gap) e[j] = 0.f;
-                if (++rloc == w) rloc = 0;
+            for (int i = 0; i < 32; i += 4) {
+                if (i < width) {
+                    const float4 L = *reinterpret_cast<const float4 *>(lse + r0 + i);
+                    float e[4];
+                    e[0] = ex2(fmaf(__uint_as_float(cur[i]), scale, -L.x));
+                    e[1] = ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -L.y));
+                    e[2] = ex2(fmaf(__uint_as_float(cur[i + 2]), scale, -L.z));
+                    e[3] = ex2(fmaf(__uint_as_float(cur[i + 3]), scale, -L.w));
+                    if (MASKED) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (rloc < pos_gap) e[j] = 0.f;
+                            if (++rloc == w) rloc = 0;
+                        }
+                    }
+                    s0 += e[0] + e[2];
+                    s1 += e[1] + e[3];
+                }
             }
         }
-        s0 += e[0] + e[2];
-        s1 += e[1] + e[3];
     }
     return s0 + s1;
 }
 
-__device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1)
+// CTA that owns item x when `items` are split evenly over `ctas` (ctas <= items).
+__device__ inline int cta_of_item(int x, int items, int ctas)
+{
+    return (int)((((int64_t)x + 1) * ctas - 1) / items);
+}
+
+__device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1,
+                                      int items, int ctas)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wg = warp >> 2, lane_base = (warp & 3) * 32;
     const int tid = threadIdx.x;                                   // 0..255
     const float scale = kLog2e * rsqrtf((float)kD);
-    const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads;
+    const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
     const int ncol_wg = sh.ncol / 2;                               // columns per warpgroup (multiple of 16)
     int cur_u = -1, buf = 0, par = 0;
     uint32_t aphase[2] = {0, 0}, ephase = 0;
     bool ok = true;
     for (int item = item0; item < item1 && ok; ++item) {
-        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, Hkv, item);
         if (it.u != cur_u) {
             if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
-            for (int r = tid; r < sh.R; r += kEpiWarps * 32) tl.lse[r] = a.lse[(int64_t)it.u * sh.Rpad + r];
+            // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
+            // left per (CTA, unit), in ascending CTA order (the same order in every CTA that needs it)
+            const int ts = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
+            const int ib = tl.seq.tiles[it.s] * Hkv + it.g * ts;
+            const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
+            for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
+                float M = -INFINITY, Z = 0.f;
+                for (int c = c_lo; c <= c_hi; ++c) {
+                    const float2 pr = a.part[(int64_t)(c + it.u) * sh.Rpad + r];
+                    if (pr.y > 0.f) {
+                        if (pr.x > M) { Z = Z * ex2(M - pr.x) + pr.y; M = pr.x; }
+                        else Z += pr.y * ex2(pr.x - M);
+                    }
+                }
+                tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;     // a row that sees nothing adds 2^(-inf) = 0
+            }
             if (!(ok = epi_sync(tl, ephase))) break;
             cur_u = it.u;
         }
@@ -520,13 +565,8 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)(wg * ncol_wg) + ((uint32_t)lane_base << 16);
             const int rbase = job * sh.ncol + wg * ncol_wg;
-            int c = 0;
-            for (; c + 32 <= ncol_wg; c += 32)
-                acc += full ? col_sum_chunk<false, 32>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap)
-                            : col_sum_chunk<true, 32>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap);
-            if (c < ncol_wg)
-                acc += full ? col_sum_chunk<false, 16>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap)
-                            : col_sum_chunk<true, 16>(taddr + c, scale, tl.lse, rbase + c, w, pos_gap);
+            acc += full ? col_sum_job<false>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap)
+                        : col_sum_job<true>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
@@ -576,12 +616,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = tl.tmem_base;
 
+    // ranges over min(grid, items) CTAs, so that every CTA that has a range has a non-empty one
     const int items = tl.seq.tiles[a.p.num_seqs] * a.p.num_kv_heads;
-    const int item0 = range_begin(blockIdx.x, items, gridDim.x), item1 = range_begin(blockIdx.x + 1, items, gridDim.x);
+    const int ctas = max(1, min((int)gridDim.x, items));
+    const bool active = (int)blockIdx.x < ctas;
+    const int item0 = active ? range_begin(blockIdx.x, items, ctas) : 0;
+    const int item1 = active ? range_begin(blockIdx.x + 1, items, ctas) : 0;
 
     if (warp < kEpiWarps) {
         if (PASS == 1) epilogue_pass1(a, tl, tmem_base, item0, item1);
-        else epilogue_pass2(a, tl, tmem_base, item0, item1);
+        else epilogue_pass2(a, tl, tmem_base, item0, item1, items, ctas);
     } else if (warp == kEpiWarps) {
         if (lane == 0) producer_loop<PASS>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1);
     } else {
@@ -595,46 +639,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     tc_fence_after();
     if (threadIdx.x == 0 && tl.abort_flag && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_TIMEOUT);
     if (warp == kEpiWarps + 1) tmem_dealloc(tmem_base, 512);
-}
-
-// L[u][row] = log2 sum over the row's visible positions of 2^y, from the per-(CTA, unit) partials.
-__global__ void score_tc_combine(TcArgs a, int ctas)
-{
-    __shared__ SeqTables seq;
-    const TcShape &sh = a.sh;
-    const int B = a.p.num_seqs, Hkv = a.p.num_kv_heads;
-    build_seq_tables(seq, a.seq_len, B);
-    const int items = seq.tiles[B] * Hkv;
-    const int64_t total = (int64_t)B * Hkv * sh.R;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int row = (int)(e % sh.R), u = (int)(e / sh.R);
-        const int s = u / Hkv, g = u % Hkv;
-        const int ts = seq.tiles[s + 1] - seq.tiles[s];
-        float L = INFINITY;                                   // a row that sees nothing contributes 2^(-inf) = 0
-        if (ts > 0) {
-            const int ib = seq.tiles[s] * Hkv + g * ts, ie = ib + ts;      // the unit's items
-            // CTAs whose ranges meet [ib, ie)
-            int c0 = (int)(((int64_t)ib * ctas) / items);
-            while (c0 > 0 && range_begin(c0, items, ctas) > ib) --c0;
-            while (c0 + 1 < ctas && range_begin(c0 + 1, items, ctas) <= ib) ++c0;
-            float m = -INFINITY;
-            // a CTA took part in the unit iff its (non-empty) range meets [ib, ie)
-            auto meets = [&](int c) {
-                const int b0 = range_begin(c, items, ctas), b1 = range_begin(c + 1, items, ctas);
-                return b1 > b0 && b1 > ib && b0 < ie;
-            };
-            for (int c = c0; c < ctas && range_begin(c, items, ctas) < ie; ++c)
-                if (meets(c)) m = fmaxf(m, a.part[(int64_t)(c + u) * sh.Rpad + row].x);
-            float z = 0.f;
-            for (int c = c0; c < ctas && range_begin(c, items, ctas) < ie; ++c) {
-                if (!meets(c)) continue;
-                const float2 pr = a.part[(int64_t)(c + u) * sh.Rpad + row];
-                if (pr.y > 0.f) z += pr.y * exp2f(pr.x - m);
-            }
-            if (z > 0.f) L = m + log2f(z);
-        }
-        a.lse[(int64_t)u * sh.Rpad + row] = L;
-    }
 }
 
 // ------------------------------------------------------------------ host -----
@@ -741,17 +745,14 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.seq_start = seq_start;
     a.seq_len = seq_len;
     a.part = reinterpret_cast<float2 *>(ws + lay.part_off);
-    a.lse = reinterpret_cast<float *>(ws + lay.lse_off);
     a.scores = scores;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;
     const size_t smem = smem_bytes(sh);
     if (smem > 232448) return cudaErrorInvalidValue;
     score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
-    const int64_t rows = (int64_t)p.num_seqs * p.num_kv_heads * sh.R;
-    score_tc_combine<<<(int)std::min<int64_t>((rows + 255) / 256, 1024), 256, 0, st>>>(a, ctas);
     score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
-    count_launches(3);
+    count_launches(2);
     return cudaGetLastError();
 }
 

@@ -99,7 +99,10 @@ __device__ inline int block_min(int x, int *buf)
 
 // Prefix scan over ranks [0, count) in the order given by `pos_of`, starting from
 // C = 0: returns the first rank count j (1-based) at which the rule is met, or
-// INT_MAX, and the sum over all `count` ranks.
+// INT_MAX, and the sum over all `count` ranks.  Each thread owns a contiguous run
+// of ranks.  The rule (an fp64 divide and square root) is evaluated once per
+// thread at the end of its run; the leftmost run whose end meets it holds the
+// crossing, and warp 0 resolves it inside that run, 32 ranks at a time.
 template <typename PosOf>
 __device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, double Cn, double T,
                                 bool search, double *dbuf, int *ibuf, double &sum)
@@ -109,16 +112,32 @@ __device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, doub
     double local = 0.0;
     for (int j = j0; j < j1; ++j) local += sq_at(v, pos_of(v, j));
     const double before = block_excl_scan<double>(local, dbuf, sum);
-    int cand = INT_MAX;
-    if (search) {
-        double C = before;
-        for (int j = j0; j < j1; ++j) {
-            C += sq_at(v, pos_of(v, j));
-            if (crossed(C, Cn, T)) { cand = j + 1; break; }
+    if (!search) return INT_MAX;
+    int hit = (j1 > j0 && crossed(before + local, Cn, T)) ? (int)threadIdx.x : INT_MAX;
+    hit = block_min(hit, ibuf);
+    if (hit == INT_MAX) return INT_MAX;
+    __syncthreads();
+    if ((int)threadIdx.x == hit) dbuf[0] = before;
+    __syncthreads();
+    const int h0 = min(count, hit * per), h1 = min(count, h0 + per);
+    int found = h1;                                   // the run's end meets the rule by construction
+    if (threadIdx.x < 32) {
+        double run = dbuf[0];
+        const int lane = threadIdx.x;
+        for (int base = h0; base < h1; base += 32) {
+            const int j = base + lane;
+            double x = j < h1 ? sq_at(v, pos_of(v, j)) : 0.0;
+            x = warp_incl_scan(x);
+            const unsigned m = __ballot_sync(0xffffffffu, j < h1 && crossed(run + x, Cn, T));
+            if (m) { found = base + __ffs(m); break; }
+            run += __shfl_sync(0xffffffffu, x, 31);
         }
-        cand = block_min(cand, ibuf);
+        if (lane == 0) ibuf[0] = found;
     }
-    return cand;
+    __syncthreads();
+    found = ibuf[0];
+    __syncthreads();
+    return found;
 }
 
 struct SelectSmem {
@@ -346,12 +365,16 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
 cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
                           int64_t total_tokens, int32_t *lengths, int64_t *offsets,
                           int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,
-                          int32_t *dev_status, cudaStream_t st)
+                          int32_t *dev_status, cudaStream_t st, bool emit)
 {
     Cut *cuts = reinterpret_cast<Cut *>(ws + lay.cut_off);
     const int U = p.num_seqs * p.num_kv_heads;
     const int sel_units = p.scope == REFREE_SCOPE_LAYER ? p.num_seqs : U;
     select_budget_kernel<<<sel_units, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts);
+    if (!emit) {               // the caller forms the offsets itself and needs no index list
+        count_launches(1);
+        return cudaGetLastError();
+    }
     const bool ranges = p.rank_mode == REFREE_RANK_POSITION || p.force_full;
     int gx = 1;
     if (ranges && kept_idx) {

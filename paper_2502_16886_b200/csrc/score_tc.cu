@@ -541,11 +541,18 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
             for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
                 float M = -INFINITY, Z = 0.f;
-                for (int c = c_lo; c <= c_hi; ++c) {
-                    const float2 pr = a.part[(int64_t)(c + it.u) * sh.Rpad + r];
-                    if (pr.y > 0.f) {
-                        if (pr.x > M) { Z = Z * ex2(M - pr.x) + pr.y; M = pr.x; }
-                        else Z += pr.y * ex2(pr.x - M);
+                for (int c0 = c_lo; c0 <= c_hi; c0 += 8) {
+                    float2 pr[8];                                  // eight independent loads in flight
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        pr[q] = (c0 + q <= c_hi) ? __ldcg(&a.part[(int64_t)(c0 + q + it.u) * sh.Rpad + r])
+                                                 : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (pr[q].y > 0.f) {
+                            if (pr[q].x > M) { Z = Z * ex2(M - pr[q].x) + pr[q].y; M = pr[q].x; }
+                            else Z += pr[q].y * ex2(pr[q].x - M);
+                        }
                     }
                 }
                 tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;     // a row that sees nothing adds 2^(-inf) = 0

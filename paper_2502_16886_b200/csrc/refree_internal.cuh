@@ -36,9 +36,9 @@ struct Workspace {
 struct Cut {
     int32_t b;          // budget (kept count)
     int32_t ties;       // score ranking: number of positions with key == tau to keep
-    uint64_t tau;       // score ranking: key threshold (bits of the fp64 squared score)
+    uint64_t tau;       // score ranking: key threshold (score bits << 32, or the fixed-point layer key)
     int32_t prot_kept;  // score ranking: protected positions kept
-    int32_t pad;
+    int32_t sbias;      // fixed-point exponent bias of the unit's squares (see select.cu)
 };
 
 Workspace workspace_layout(const refree_params &p, int64_t total_tokens);

@@ -1,19 +1,27 @@
 // Steps S4-S6: ranking, the threshold-free stopping rule and the kept set.
 //
-// For one unit with squares sq_i = (double)a'_i^2 (exact: a' is fp32) and ranked
-// order pi, the rule is the cumulative form of Eq. 1 (Eq. 3; Algorithm 1 Square,
-// Reorder, Cumsum, Sqrt, ratio, Where):
-//     C_j = sum_{t<=j} sq[pi_t],  j* = leftmost j with 1 - sqrt(C_j / C_n) < T,
-// all of it in fp64.  The budget is b = max(j*, floor); the kept set is the first
-// b ranked positions, emitted in ascending position order.
+// For one unit with squares sq_i = a'_i^2 and ranked order pi, the rule is the
+// cumulative form of Eq. 1 (Eq. 3; Algorithm 1 Square, Reorder, Cumsum, Sqrt,
+// ratio, Where):
+//     C_j = sum_{t<=j} sq[pi_t],  j* = leftmost j with 1 - sqrt(C_j / C_n) < T.
+// The budget is b = max(j*, floor); the kept set is the first b ranked positions,
+// emitted in ascending position order.
+//
+// Arithmetic.  fp64 is a slow pipe on this GPU, so the sums are integers: the
+// square of an fp32 score is the exact 48-bit product of its mantissa with
+// itself, shifted to a per-unit fixed point in which C_n lies in [2^60, 2^61)
+// (bits below the unit are dropped: at most n * 2^-60 of C_n in total).  Integer
+// sums do not depend on the order of addition, so budgets are deterministic.
+// The rule itself is applied as C_j >= C_min, where
+//     1 - sqrt(C/C_n) < T  <=>  C_n - C < C_n * T * (2 - T)
+// and C_min is placed once per unit with a handful of fp64 operations.
 //
 // Position ranking (Section 3.2) needs no sort: the order is the m leading
 // positions, then the rest from the end backwards, so C_j is a block-wide prefix
 // scan over a closed-form order.  Score ranking (Section 4.4) needs the order by
-// decreasing score; instead of sorting, a radix descent over the 64-bit keys
-// (8 bits per level) finds the key at which the cumulative sum crosses, using
-// per-digit histograms of counts and of fixed-point sums of squares.  Integer
-// sums make the result independent of the order in which threads add.
+// decreasing score; instead of sorting, a radix descent over the keys (8 bits per
+// level) finds the key at which the cumulative sum crosses, using per-digit
+// histograms of counts and of sums of squares.
 #include <algorithm>
 
 #include "refree_internal.cuh"
@@ -23,38 +31,50 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
-
-__device__ inline bool crossed(double C, double Cn, double T)
-{
-    return Cn > 0.0 && (1.0 - __dsqrt_rn(__ddiv_rn(C, Cn))) < T;
-}
+typedef unsigned long long u64;
 
 struct UnitView {
     const float *sc;        // scores of head 0 (layer scope) or of the unit's head, at the sequence start
     int64_t head_stride;    // distance between heads in the score array
     int heads;              // heads whose squares add up (1 in head scope)
     int n, lead, w_eff;
+    int sbias;              // fixed point: a^2 * 2^S = mantissa^2 * 2^(2 * exponent_field + sbias)
 };
 
-__device__ inline double sq_at(const UnitView &v, int i)
+__device__ inline uint32_t mag_bits(float a) { return __float_as_uint(a) & 0x7fffffffu; }
+
+// floor(a^2 * 2^S) from the bits of |a|; non-finite values count as zero
+__device__ inline u64 sq_fixed(uint32_t bits, int sbias)
 {
-    double acc = 0.0;
-    for (int h = 0; h < v.heads; ++h) {
-        const double a = (double)v.sc[(int64_t)h * v.head_stride + i];
-        acc += a * a;
-    }
+    const uint32_t e = bits >> 23;
+    if (e == 255u) return 0ull;
+    const uint32_t m = (bits & 0x7fffffu) | (e ? 0x800000u : 0u);
+    const u64 mm = (u64)m * m;                                   // exact, below 2^48
+    const int sh = 2 * (int)(e ? e : 1u) + sbias;
+    if (sh >= 0) return sh < 16 ? mm << sh : ~0ull >> 2;
+    return -sh < 48 ? mm >> -sh : 0ull;
+}
+
+__device__ inline u64 sq_at(const UnitView &v, int i)
+{
+    u64 acc = 0;
+    for (int h = 0; h < v.heads; ++h) acc += sq_fixed(mag_bits(v.sc[(int64_t)h * v.head_stride + i]), v.sbias);
     return acc;
 }
 
-// position of protected rank j: leading positions, then (score ranking) the window
-__device__ inline int pos_of_rank_position_mode(const UnitView &v, int j)
+// sort key of an unprotected position: larger key = ranked earlier
+__device__ inline u64 key_at(const UnitView &v, int i)
 {
-    return j < v.lead ? j : v.n - 1 - (j - v.lead);
+    if (v.heads == 1) return (u64)mag_bits(v.sc[i]) << 32;       // a' >= 0: its bits order like its square
+    return sq_at(v, i);
 }
-__device__ inline int pos_of_protected_rank(const UnitView &v, int j)
-{
-    return j < v.lead ? j : v.n - v.w_eff + (j - v.lead);
-}
+
+struct PosRank {     // position ranking: leading positions, then from the end backwards
+    __device__ int operator()(const UnitView &v, int j) const { return j < v.lead ? j : v.n - 1 - (j - v.lead); }
+};
+struct ProtRank {    // protected prefix of the score ranking: leading positions, then the window
+    __device__ int operator()(const UnitView &v, int j) const { return j < v.lead ? j : v.n - v.w_eff + (j - v.lead); }
+};
 
 template <typename Tv> __device__ inline Tv warp_incl_scan(Tv x)
 {
@@ -86,75 +106,119 @@ template <typename Tv> __device__ inline Tv block_excl_scan(Tv x, Tv *buf, Tv &t
     return buf[warp] + inc - x;
 }
 
-__device__ inline int block_min(int x, int *buf)
+template <typename Tv, typename Op> __device__ inline Tv block_reduce(Tv x, Tv *buf, Op op)
 {
-    for (int o = 16; o; o >>= 1) x = min(x, __shfl_xor_sync(0xffffffffu, x, o));
+    for (int o = 16; o; o >>= 1) x = op(x, __shfl_xor_sync(0xffffffffu, x, o));
     __syncthreads();
     if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = x;
     __syncthreads();
-    int r = buf[0];
-    for (int wv = 1; wv < kWarps; ++wv) r = min(r, buf[wv]);
+    Tv r = buf[0];
+    for (int wv = 1; wv < kWarps; ++wv) r = op(r, buf[wv]);
     return r;
 }
+struct MinOp { __device__ int operator()(int a, int b) const { return min(a, b); } };
+struct MaxOpU { __device__ uint32_t operator()(uint32_t a, uint32_t b) const { return max(a, b); } };
+struct AddOpF { __device__ float operator()(float a, float b) const { return a + b; } };
 
 // Prefix scan over ranks [0, count) in the order given by `pos_of`, starting from
-// C = 0: returns the first rank count j (1-based) at which the rule is met, or
-// INT_MAX, and the sum over all `count` ranks.  Each thread owns a contiguous run
-// of ranks.  The rule (an fp64 divide and square root) is evaluated once per
-// thread at the end of its run; the leftmost run whose end meets it holds the
-// crossing, and warp 0 resolves it inside that run, 32 ranks at a time.
+// C = 0: returns the first rank count j (1-based) with C_j >= c_min, or INT_MAX,
+// and the sum over all `count` ranks.  Each thread owns a contiguous run of ranks;
+// the leftmost run whose end reaches c_min holds the crossing, and warp 0 resolves
+// it inside that run, 32 ranks at a time.
 template <typename PosOf>
-__device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, double Cn, double T,
-                                bool search, double *dbuf, int *ibuf, double &sum)
+__device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, u64 c_min, bool search,
+                                u64 *ubuf, int *ibuf, u64 &sum)
 {
     const int per = ceil_div(count, kThreads);
     const int j0 = min(count, (int)threadIdx.x * per), j1 = min(count, j0 + per);
-    double local = 0.0;
+    u64 local = 0;
     for (int j = j0; j < j1; ++j) local += sq_at(v, pos_of(v, j));
-    const double before = block_excl_scan<double>(local, dbuf, sum);
+    const u64 before = block_excl_scan<u64>(local, ubuf, sum);
     if (!search) return INT_MAX;
-    int hit = (j1 > j0 && crossed(before + local, Cn, T)) ? (int)threadIdx.x : INT_MAX;
-    hit = block_min(hit, ibuf);
+    int hit = (j1 > j0 && before + local >= c_min) ? (int)threadIdx.x : INT_MAX;
+    hit = block_reduce<int>(hit, ibuf, MinOp());
     if (hit == INT_MAX) return INT_MAX;
     __syncthreads();
-    if ((int)threadIdx.x == hit) dbuf[0] = before;
+    if ((int)threadIdx.x == hit) ubuf[0] = before;
     __syncthreads();
     const int h0 = min(count, hit * per), h1 = min(count, h0 + per);
-    int found = h1;                                   // the run's end meets the rule by construction
     if (threadIdx.x < 32) {
-        double run = dbuf[0];
+        u64 run = ubuf[0];
         const int lane = threadIdx.x;
+        int found = h1;
         for (int base = h0; base < h1; base += 32) {
             const int j = base + lane;
-            double x = j < h1 ? sq_at(v, pos_of(v, j)) : 0.0;
+            u64 x = j < h1 ? sq_at(v, pos_of(v, j)) : 0ull;
             x = warp_incl_scan(x);
-            const unsigned m = __ballot_sync(0xffffffffu, j < h1 && crossed(run + x, Cn, T));
+            const unsigned m = __ballot_sync(0xffffffffu, j < h1 && run + x >= c_min);
             if (m) { found = base + __ffs(m); break; }
             run += __shfl_sync(0xffffffffu, x, 31);
         }
         if (lane == 0) ibuf[0] = found;
     }
     __syncthreads();
-    found = ibuf[0];
+    const int found = ibuf[0];
     __syncthreads();
     return found;
 }
 
 struct SelectSmem {
-    double dbuf[kWarps + 1];
+    u64 ubuf[kWarps + 1];
     int ibuf[kWarps + 1];
+    float fbuf[kWarps + 1];
     unsigned int hcnt[256];
-    unsigned long long hsum[256];
+    u64 hsum[256];
     int pack;
+    u64 c_min;
     // radix state
-    unsigned long long prefix, above_sum;
+    u64 prefix, above_sum;
     unsigned int above_cnt;
     int digit;
 };
 
+// Fixed point of a unit: returns false when every score is zero (C_n = 0).
+__device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *dev_status)
+{
+    uint32_t mx = 0;
+    bool bad = false;
+    for (int h = 0; h < v.heads; ++h)
+        for (int i = threadIdx.x; i < v.n; i += kThreads) {
+            const uint32_t b = mag_bits(v.sc[(int64_t)h * v.head_stride + i]);
+            if ((b >> 23) == 255u) bad = true; else mx = max(mx, b);
+        }
+    if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
+    mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
+    if (mx == 0u) return false;
+    const int emax = max(1, (int)(mx >> 23));
+    // approximate sum of squares of the scores scaled into [0, 2): only its binary order of magnitude is used
+    const float f = ldexpf(1.0f, 127 - emax);
+    float acc = 0.f;
+    for (int h = 0; h < v.heads; ++h)
+        for (int i = threadIdx.x; i < v.n; i += kThreads) {
+            const uint32_t b = mag_bits(v.sc[(int64_t)h * v.head_stride + i]);
+            const float a = ((b >> 23) == 255u) ? 0.f : __uint_as_float(b) * f;
+            acc = fmaf(a, a, acc);
+        }
+    acc = block_reduce<float>(acc, sm.fbuf, AddOpF());
+    // C_n = acc * 2^(2 (emax - 127)); put C_n * 2^S in [2^60, 2^61)
+    const int S = 60 - ilogbf(fmaxf(acc, 0.25f)) - 2 * (emax - 127);
+    v.sbias = S - 300;
+    return true;
+}
+
+// Smallest fixed-point C with 1 - sqrt(C / Cn) < T, i.e. Cn - C < Cn * T * (2 - T); ~0 when there is none.
+__device__ inline u64 crossing_level(u64 Cn, double T)
+{
+    const double lim = (double)Cn * (T * (2.0 - T));
+    const double c = ceil(lim);
+    if (!(c >= 1.0)) return ~0ull;                 // T = 0: never met
+    const u64 dmax = (u64)c - 1ull;                // largest dropped mass that still meets the rule
+    return dmax >= Cn ? 0ull : Cn - dmax;
+}
+
 __global__ void __launch_bounds__(kThreads)
 select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_len,
-                     int64_t total_tokens, int32_t *lengths, Cut *cuts)
+                     int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status)
 {
     __shared__ SelectSmem sm;
     const int Hkv = p.num_kv_heads;
@@ -168,7 +232,6 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     }
     __syncthreads();
     const int n = max(seq_len[s], 0);
-    const double T = (double)p.threshold;
     UnitView v;
     v.sc = scores + (int64_t)g * total_tokens + sm.pack;
     v.head_stride = total_tokens;
@@ -176,93 +239,85 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     v.n = n;
     v.w_eff = min(p.window, n);
     v.lead = min(p.sink, n);
+    v.sbias = 0;
     const int floor_b = p.keep_window ? min(n, v.lead + v.w_eff) : min(n, 1);
 
     Cut cut;
-    cut.b = n; cut.ties = 0; cut.tau = 0; cut.prot_kept = 0; cut.pad = 0;
+    cut.b = n; cut.ties = 0; cut.tau = 0; cut.prot_kept = 0; cut.sbias = 0;
 
-    if (n > 0 && !p.force_full) {
+    if (n > 0 && !p.force_full && choose_fixed_point(v, sm, dev_status)) {
+        cut.sbias = v.sbias;
+        u64 Cn, dummy;
+        {   // C_n over every position (the order does not matter for an integer sum)
+            UnitView all = v; all.lead = n; all.w_eff = 0;
+            scan_find(all, n, ProtRank(), 0ull, false, sm.ubuf, sm.ibuf, Cn);
+        }
+        if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
+        __syncthreads();
+        const u64 c_min = sm.c_min;
         if (p.rank_mode == REFREE_RANK_POSITION) {
-            double Cn, dummy;
-            scan_find(v, n, pos_of_rank_position_mode, 0.0, T, false, sm.dbuf, sm.ibuf, Cn);
-            const int j = scan_find(v, n, pos_of_rank_position_mode, Cn, T, true, sm.dbuf, sm.ibuf, dummy);
-            const int jstar = (j == INT_MAX) ? n : j;
-            cut.b = max(jstar, floor_b);
+            const int j = scan_find(v, n, PosRank(), c_min, true, sm.ubuf, sm.ibuf, dummy);
+            cut.b = max(j == INT_MAX ? n : j, floor_b);
         } else {
             // score ranking: when the protected prefix covers the sequence the order is 0..n-1
             if (v.lead + v.w_eff >= n) { v.lead = n; v.w_eff = 0; }
             const int prot = v.lead + v.w_eff;
-            double Cn, Sprot;
-            // C_n over every position (position order is as good as any for the total)
-            {
-                UnitView all = v; all.lead = n; all.w_eff = 0;
-                scan_find(all, n, pos_of_protected_rank, 0.0, T, false, sm.dbuf, sm.ibuf, Cn);
-            }
-            const int jp = scan_find(v, prot, pos_of_protected_rank, Cn, T, true, sm.dbuf, sm.ibuf, Sprot);
+            u64 Sprot;
+            const int jp = scan_find(v, prot, ProtRank(), c_min, true, sm.ubuf, sm.ibuf, Sprot);
             int jstar = n;
             cut.prot_kept = prot;
             cut.tau = 0ull;                       // keep every unprotected position ...
             cut.ties = INT_MAX;                   // ... unless a crossing is found below
             if (jp != INT_MAX) {
                 jstar = jp;
-            } else if (Cn > 0.0 && prot < n) {
-                // fixed point with C_n * 2^e in [2^61, 2^62)
-                const int e = 61 - ilogb(Cn);
+            } else if (prot < n && c_min != ~0ull) {
+                const u64 need = c_min - Sprot;   // mass still missing after the protected prefix (> 0)
                 if (threadIdx.x == 0) { sm.prefix = 0ull; sm.above_sum = 0ull; sm.above_cnt = 0u; }
+                const int levels = v.heads == 1 ? 4 : 8;
                 bool any = true;
-                for (int level = 0; level < 8 && any; ++level) {
+                for (int level = 0; level < levels && any; ++level) {
                     const int shift = 56 - 8 * level;
                     for (int t = threadIdx.x; t < 256; t += kThreads) { sm.hcnt[t] = 0u; sm.hsum[t] = 0ull; }
                     __syncthreads();
-                    const unsigned long long prefix = sm.prefix;
+                    const u64 prefix = sm.prefix;
                     for (int i = v.lead + threadIdx.x; i < n - v.w_eff; i += kThreads) {
-                        const double x = sq_at(v, i);
-                        const unsigned long long key = (unsigned long long)__double_as_longlong(x);
+                        const u64 key = key_at(v, i);
                         if (level == 0 || (key >> (shift + 8)) == prefix) {
                             const int dgt = (int)((key >> shift) & 255ull);
                             atomicAdd(&sm.hcnt[dgt], 1u);
-                            atomicAdd(&sm.hsum[dgt], __double2ull_rd(ldexp(x, e)));
+                            atomicAdd(&sm.hsum[dgt], v.heads == 1 ? sq_at(v, i) : key);
                         }
                     }
                     __syncthreads();
                     // inclusive sums from the top digit down; thread t owns digit 255 - t
-                    unsigned long long mysum = 0ull, tot_s;
+                    u64 mysum = 0ull, tot_s;
                     unsigned int mycnt = 0u, tot_c;
                     if (threadIdx.x < 256) { mysum = sm.hsum[255 - threadIdx.x]; mycnt = sm.hcnt[255 - threadIdx.x]; }
-                    const unsigned long long abv_s = block_excl_scan<unsigned long long>(mysum, (unsigned long long *)sm.dbuf, tot_s);
+                    const u64 abv_s = block_excl_scan<u64>(mysum, sm.ubuf, tot_s);
                     const unsigned int abv_c = block_excl_scan<unsigned int>(mycnt, (unsigned int *)sm.ibuf, tot_c);
                     int cand = INT_MAX;
-                    if (threadIdx.x < 256 && mycnt > 0u) {
-                        const double C = Sprot + ldexp((double)(sm.above_sum + abv_s + mysum), -e);
-                        if (crossed(C, Cn, T)) cand = threadIdx.x;
-                    }
-                    cand = block_min(cand, sm.ibuf);
+                    if (threadIdx.x < 256 && mycnt > 0u && sm.above_sum + abv_s + mysum >= need) cand = threadIdx.x;
+                    cand = block_reduce<int>(cand, sm.ibuf, MinOp());
                     if (cand == INT_MAX) {
                         any = false;              // the rule is never met: keep all
-                    } else {
-                        if ((int)threadIdx.x == cand) {
-                            sm.prefix = (prefix << 8) | (unsigned long long)(255 - cand);
-                            sm.above_sum += abv_s;
-                            sm.above_cnt += abv_c;
-                            sm.digit = (int)mycnt;
-                        }
+                    } else if ((int)threadIdx.x == cand) {
+                        sm.prefix = (prefix << 8) | (u64)(255 - cand);
+                        sm.above_sum += abv_s;
+                        sm.above_cnt += abv_c;
+                        sm.digit = (int)mycnt;
                     }
                     __syncthreads();
                 }
                 if (any) {
-                    // sm.prefix is the full key at which the sum crosses; sm.digit of them tie
-                    const unsigned long long tau = sm.prefix;
-                    const int ties_total = sm.digit;
-                    const unsigned long long f = __double2ull_rd(ldexp(__longlong_as_double((long long)tau), e));
-                    int lo = 1, hi = ties_total;   // smallest t with the rule met; t = hi is known to meet it
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        const double C = Sprot + ldexp((double)(sm.above_sum + (unsigned long long)mid * f), -e);
-                        if (crossed(C, Cn, T)) hi = mid; else lo = mid + 1;
-                    }
-                    jstar = prot + (int)sm.above_cnt + lo;
+                    // sm.prefix is the key at which the sum crosses; sm.digit positions share it
+                    const u64 tau = v.heads == 1 ? sm.prefix << 32 : sm.prefix;
+                    const u64 f = v.heads == 1 ? sq_fixed((uint32_t)sm.prefix, v.sbias) : tau;
+                    const u64 miss = need - sm.above_sum;           // > 0: the digits above did not reach it
+                    u64 t = f ? (miss + f - 1) / f : 1ull;
+                    t = max(1ull, min(t, (u64)sm.digit));
+                    jstar = prot + (int)sm.above_cnt + (int)t;
                     cut.tau = tau;
-                    cut.ties = lo;
+                    cut.ties = (int)t;
                 }
             }
             cut.b = max(jstar, floor_b);
@@ -335,6 +390,7 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     v.head_stride = total_tokens;
     v.heads = layer ? Hkv : 1;
     v.n = n; v.lead = lead; v.w_eff = w_eff;
+    v.sbias = cut.sbias;
     int base = 0, tie_base = 0;
     for (int i0 = 0; i0 < n; i0 += kThreads) {
         const int i = i0 + threadIdx.x;
@@ -345,7 +401,7 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
             } else if (i >= n - w_eff) {
                 keep = lead + (i - (n - w_eff)) < cut.prot_kept;
             } else {
-                const unsigned long long key = (unsigned long long)__double_as_longlong(sq_at(v, i));
+                const u64 key = key_at(v, i);
                 keep = key > cut.tau;
                 tie = key == cut.tau;
             }
@@ -370,7 +426,7 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     Cut *cuts = reinterpret_cast<Cut *>(ws + lay.cut_off);
     const int U = p.num_seqs * p.num_kv_heads;
     const int sel_units = p.scope == REFREE_SCOPE_LAYER ? p.num_seqs : U;
-    select_budget_kernel<<<sel_units, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts);
+    select_budget_kernel<<<sel_units, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
     if (!emit) {               // the caller forms the offsets itself and needs no index list
         count_launches(1);
         return cudaGetLastError();
@@ -378,7 +434,7 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     const bool ranges = p.rank_mode == REFREE_RANK_POSITION || p.force_full;
     int gx = 1;
     if (ranges && kept_idx) {
-        const int64_t per_unit = std::max<int64_t>(1, total_tokens / max(1, p.num_seqs));
+        const int64_t per_unit = std::max<int64_t>(1, total_tokens / std::max(1, p.num_seqs));
         gx = (int)std::min<int64_t>(16, (per_unit + 4 * kThreads - 1) / (4 * kThreads));
     }
     emit_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, offsets,

@@ -120,37 +120,56 @@ struct MinOp { __device__ int operator()(int a, int b) const { return min(a, b);
 struct MaxOpU { __device__ uint32_t operator()(uint32_t a, uint32_t b) const { return max(a, b); } };
 struct AddOpF { __device__ float operator()(float a, float b) const { return a + b; } };
 
-// Prefix scan over ranks [0, count) in the order given by `pos_of`, starting from
-// C = 0: returns the first rank count j (1-based) with C_j >= c_min, or INT_MAX,
-// and the sum over all `count` ranks.  Each thread owns a contiguous run of ranks;
-// the leftmost run whose end reaches c_min holds the crossing, and warp 0 resolves
-// it inside that run, 32 ranks at a time.
+// Ranks [0, count) in the order given by `pos_of` are split into one contiguous
+// segment per warp; inside a segment the lanes interleave, so every load is a
+// coalesced 128-byte line.  seg_totals leaves the exclusive prefix of the warp
+// sums in wpre[0..kWarps) and the grand total in wpre[kWarps].
+__device__ inline int seg_len(int count) { return ceil_div(ceil_div(count, kWarps), 32) * 32; }
+
 template <typename PosOf>
-__device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, u64 c_min, bool search,
-                                u64 *ubuf, int *ibuf, u64 &sum)
+__device__ inline u64 seg_totals(const UnitView &v, int count, PosOf pos_of, u64 *wpre)
 {
-    const int per = ceil_div(count, kThreads);
-    const int j0 = min(count, (int)threadIdx.x * per), j1 = min(count, j0 + per);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int seg = seg_len(count);
+    const int w0 = min(count, warp * seg), w1 = min(count, w0 + seg);
     u64 local = 0;
-    for (int j = j0; j < j1; ++j) local += sq_at(v, pos_of(v, j));
-    const u64 before = block_excl_scan<u64>(local, ubuf, sum);
-    if (!search) return INT_MAX;
-    int hit = (j1 > j0 && before + local >= c_min) ? (int)threadIdx.x : INT_MAX;
-    hit = block_reduce<int>(hit, ibuf, MinOp());
-    if (hit == INT_MAX) return INT_MAX;
+    for (int j = w0 + lane; j < w1; j += 32) local += sq_at(v, pos_of(v, j));
+    for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
     __syncthreads();
-    if ((int)threadIdx.x == hit) ubuf[0] = before;
+    if (lane == 0) wpre[warp] = local;
     __syncthreads();
-    const int h0 = min(count, hit * per), h1 = min(count, h0 + per);
-    if (threadIdx.x < 32) {
-        u64 run = ubuf[0];
-        const int lane = threadIdx.x;
-        int found = h1;
-        for (int base = h0; base < h1; base += 32) {
+    if (warp == 0) {
+        const u64 x = wpre[lane];
+        const u64 inc = warp_incl_scan(x);
+        wpre[lane] = inc - x;
+        if (lane == 31) wpre[kWarps] = inc;
+    }
+    __syncthreads();
+    return wpre[kWarps];
+}
+
+// First rank count j (1-based) with C_j >= c_min, or INT_MAX, given the warp
+// prefixes of seg_totals: the first warp whose segment end reaches c_min holds
+// the crossing and resolves it 32 ranks at a time.
+template <typename PosOf>
+__device__ inline int seg_find(const UnitView &v, int count, PosOf pos_of, u64 c_min, const u64 *wpre, int *ibuf)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int seg = seg_len(count);
+    const int w0 = min(count, warp * seg), w1 = min(count, w0 + seg);
+    const u64 end = warp + 1 < kWarps ? wpre[warp + 1] : wpre[kWarps];
+    const bool first_hit = w1 > w0 && end >= c_min && wpre[warp] < c_min;   // prefixes are monotone: at most one warp
+    __syncthreads();
+    if (threadIdx.x == 0) ibuf[0] = INT_MAX;
+    __syncthreads();
+    if (first_hit) {
+        u64 run = wpre[warp];
+        int found = w1;
+        for (int base = w0; base < w1; base += 32) {
             const int j = base + lane;
-            u64 x = j < h1 ? sq_at(v, pos_of(v, j)) : 0ull;
+            u64 x = j < w1 ? sq_at(v, pos_of(v, j)) : 0ull;
             x = warp_incl_scan(x);
-            const unsigned m = __ballot_sync(0xffffffffu, j < h1 && run + x >= c_min);
+            const unsigned m = __ballot_sync(0xffffffffu, j < w1 && run + x >= c_min);
             if (m) { found = base + __ffs(m); break; }
             run += __shfl_sync(0xffffffffu, x, 31);
         }
@@ -163,6 +182,7 @@ __device__ inline int scan_find(const UnitView &v, int count, PosOf pos_of, u64 
 }
 
 struct SelectSmem {
+    u64 wpre[kWarps + 1];
     u64 ubuf[kWarps + 1];
     int ibuf[kWarps + 1];
     float fbuf[kWarps + 1];
@@ -247,23 +267,27 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
 
     if (n > 0 && !p.force_full && choose_fixed_point(v, sm, dev_status)) {
         cut.sbias = v.sbias;
-        u64 Cn, dummy;
-        {   // C_n over every position (the order does not matter for an integer sum)
-            UnitView all = v; all.lead = n; all.w_eff = 0;
-            scan_find(all, n, ProtRank(), 0ull, false, sm.ubuf, sm.ibuf, Cn);
-        }
-        if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
-        __syncthreads();
-        const u64 c_min = sm.c_min;
         if (p.rank_mode == REFREE_RANK_POSITION) {
-            const int j = scan_find(v, n, PosRank(), c_min, true, sm.ubuf, sm.ibuf, dummy);
+            // one pass in rank order gives C_n and the warp prefixes the search needs
+            const u64 Cn = seg_totals(v, n, PosRank(), sm.wpre);
+            if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
+            __syncthreads();
+            const int j = seg_find(v, n, PosRank(), sm.c_min, sm.wpre, sm.ibuf);
             cut.b = max(j == INT_MAX ? n : j, floor_b);
         } else {
             // score ranking: when the protected prefix covers the sequence the order is 0..n-1
             if (v.lead + v.w_eff >= n) { v.lead = n; v.w_eff = 0; }
             const int prot = v.lead + v.w_eff;
-            u64 Sprot;
-            const int jp = scan_find(v, prot, ProtRank(), c_min, true, sm.ubuf, sm.ibuf, Sprot);
+            u64 Cn;
+            {   // C_n over every position (the order does not matter for an integer sum)
+                UnitView all = v; all.lead = n; all.w_eff = 0;
+                Cn = seg_totals(all, n, ProtRank(), sm.wpre);
+            }
+            if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
+            __syncthreads();
+            const u64 c_min = sm.c_min;
+            const u64 Sprot = seg_totals(v, prot, ProtRank(), sm.wpre);
+            const int jp = seg_find(v, prot, ProtRank(), c_min, sm.wpre, sm.ibuf);
             int jstar = n;
             cut.prot_kept = prot;
             cut.tau = 0ull;                       // keep every unprotected position ...

@@ -109,11 +109,18 @@ __device__ inline void tmem_dealloc(uint32_t taddr, uint32_t cols)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+// The two shared-memory descriptors are passed as their low words (start address
+// and leading offset, see desc_lo) plus the common high word: one thread issues
+// every MMA of the CTA, so the issue path is kept to a few instructions.
+__device__ inline void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                 uint32_t accumulate)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+                 "setp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 da, {%1, %3};\n\t"
+                 "mov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 // The mbarrier receives one arrival once every MMA issued so far by this thread has completed.
 __device__ inline void umma_commit(uint64_t *bar)
@@ -153,16 +160,12 @@ __device__ inline float ex2(float x)
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B
 // apart, groups of 8 rows 1024 B apart (the layout TMA writes with SWIZZLE_128B).
-__device__ inline uint64_t make_desc(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);          // start address
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset: 8 rows * 128 B
-    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
-    return d;
-}
+// Low word: start address / 16 in bits 0-13, leading byte offset (unused with
+// swizzle) in bits 16-29.  A byte offset o (multiple of 16) inside the operand
+// adds o / 16 to the low word.  High word: stride byte offset / 16 in bits 0-13,
+// descriptor version 1 in bits 14-15, swizzle mode 2 (128 B) in bits 29-31.
+__device__ inline uint32_t desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
 __host__ __device__ inline uint32_t make_idesc(int n)
 {
@@ -293,7 +296,8 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
                                 uint32_t tmem_base, int item0, int item1)
 {
     const TcShape &sh = a.sh;
-    const uint32_t q_addr = smem_u32(smem_q), k_addr = smem_u32(smem_k);
+    const uint32_t q_lo = desc_lo(smem_u32(smem_q)), k_lo = desc_lo(smem_u32(smem_k));
+    const uint32_t q_half = (uint32_t)(sh.Rpad * 128) >> 4;      // distance between the two 64-column halves of Q
     const uint32_t idesc1 = make_idesc(kTile), idesc2 = make_idesc(sh.ncol);
     int cur_u = -1, stage = 0, buf = 0;
     uint32_t kphase = 0, qphase = 0, aphase[2] = {0, 0};
@@ -312,7 +316,7 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
         ok = mbar_wait(&tl.k_full[stage], kphase, &tl.abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t kt = k_addr + (uint32_t)stage * kTileBytes;
+        const uint32_t kt_lo = k_lo + (uint32_t)stage * (kTileBytes >> 4);
         const int jobs = PASS == 1 ? sh.jobs1 : sh.nb;
         for (int job = 0; job < jobs && ok; ++job) {
             ok = mbar_wait(&tl.acc_empty[buf], aphase[buf] ^ 1, &tl.abort_flag);
@@ -323,20 +327,20 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
                 for (int half_acc = 0; half_acc < 2; ++half_acc) {
                     const int rb = 2 * job + half_acc;
                     if (rb >= sh.rblocks) break;
+                    const uint32_t qa = q_lo + (uint32_t)rb * (kHalfBytes >> 4);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t h = kk >> 2, ko = (kk & 3) * 32;
-                        umma_bf16(d0 + half_acc * 128,
-                                  make_desc(q_addr + h * sh.Rpad * 128 + rb * kHalfBytes + ko),
-                                  make_desc(kt + h * kHalfBytes + ko), idesc1, kk > 0);
+                        const uint32_t h = kk >> 2, ko = (kk & 3) * 2;          // 32 bytes per K step of 16
+                        umma_bf16(d0 + half_acc * 128, qa + h * q_half + ko, kt_lo + h * (kHalfBytes >> 4) + ko,
+                                  kDescHi, idesc1, kk > 0);
                     }
                 }
             } else {
+                const uint32_t qb = q_lo + (uint32_t)job * (uint32_t)(sh.ncol * 128 >> 4);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t h = kk >> 2, ko = (kk & 3) * 32;
-                    umma_bf16(d0, make_desc(kt + h * kHalfBytes + ko),
-                              make_desc(q_addr + h * sh.Rpad * 128 + job * sh.ncol * 128 + ko), idesc2, kk > 0);
+                    const uint32_t h = kk >> 2, ko = (kk & 3) * 2;
+                    umma_bf16(d0, kt_lo + h * (kHalfBytes >> 4) + ko, qb + h * q_half + ko, kDescHi, idesc2, kk > 0);
                 }
             }
             umma_commit(&tl.acc_full[buf]);
@@ -607,6 +611,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     TcSmemTail &tl = *reinterpret_cast<TcSmemTail *>(smem_k + (size_t)sh.stages * kTileBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    if (threadIdx.x == kEpiWarps * 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapq) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapk) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) { mbar_init(&tl.k_full[s], 1); mbar_init(&tl.k_empty[s], 1); }
         mbar_init(&tl.q_full, 1);

@@ -52,6 +52,7 @@ inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; 
 struct SeqTables {
     int32_t pack[kMaxSeqs + 1];   // positions before sequence s in the packed score array
     int32_t tiles[kMaxSeqs + 1];  // scoring tiles before sequence s
+    int32_t len[kMaxSeqs];        // copy of seq_len (clamped at 0)
 };
 
 __device__ inline void build_seq_tables(SeqTables &t, const int32_t *seq_len, int B)
@@ -62,6 +63,7 @@ __device__ inline void build_seq_tables(SeqTables &t, const int32_t *seq_len, in
             t.pack[s] = a;
             t.tiles[s] = b;
             const int n = max(seq_len[s], 0);
+            t.len[s] = n;
             a += n;
             b += ceil_div(n, kTile);
         }

@@ -191,16 +191,27 @@ struct TcSmemTail {
     alignas(16) float stage[2][2][kTile];     // pass 2: per item parity, per warpgroup partial column sums
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
     SeqTables seq;
+    int32_t start[kMaxSeqs];                  // copy of seq_start
 };
 
 struct ItemTc {
     int u, s, g, n, tile_start, tok0, pack;
+    int tile, ntiles;      // tile index inside the sequence, tiles of the sequence
 };
 
-__device__ inline ItemTc decode_item_tc(const SeqTables &t, const int32_t *seq_start, const int32_t *seq_len,
-                                        int B, int Hkv, int item)
+__device__ inline void fill_seq_fields(ItemTc &it, const TcSmemTail &tl, int Hkv)
 {
-    // items are ordered (sequence, head, tile): a CTA's consecutive items mostly share a unit
+    it.u = it.s * Hkv + it.g;
+    it.n = tl.seq.len[it.s];
+    it.tok0 = tl.start[it.s];
+    it.pack = tl.seq.pack[it.s];
+    it.tile_start = it.tile * kTile;
+}
+
+// Items are ordered (sequence, head, tile): a CTA's consecutive items mostly share a unit.
+__device__ inline ItemTc decode_item_tc(const TcSmemTail &tl, int B, int Hkv, int item)
+{
+    const SeqTables &t = tl.seq;
     int lo = 0, hi = B;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -208,15 +219,29 @@ __device__ inline ItemTc decode_item_tc(const SeqTables &t, const int32_t *seq_s
     }
     ItemTc it;
     it.s = lo;
-    const int ts = t.tiles[lo + 1] - t.tiles[lo];
+    it.ntiles = t.tiles[lo + 1] - t.tiles[lo];
     const int rem = item - t.tiles[lo] * Hkv;
-    it.g = rem / ts;
-    it.tile_start = (rem % ts) * kTile;
-    it.u = lo * Hkv + it.g;
-    it.n = seq_len[lo];
-    it.tok0 = seq_start[lo];
-    it.pack = t.pack[lo];
+    it.g = rem / it.ntiles;
+    it.tile = rem % it.ntiles;
+    fill_seq_fields(it, tl, Hkv);
     return it;
+}
+
+// The item after `it` in the same order, without searching or dividing.
+__device__ inline void next_item_tc(ItemTc &it, const TcSmemTail &tl, int B, int Hkv)
+{
+    if (++it.tile < it.ntiles) {
+        it.tile_start += kTile;
+        return;
+    }
+    it.tile = 0;
+    if (++it.g == Hkv) {
+        it.g = 0;
+        do { ++it.s; } while (it.s < B - 1 && tl.seq.tiles[it.s + 1] == tl.seq.tiles[it.s]);
+        if (it.s >= B) it.s = B - 1;                 // past the end: never used, kept in range
+        it.ntiles = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
+    }
+    fill_seq_fields(it, tl, Hkv);
 }
 
 // first item of CTA c when `items` are split evenly over `ctas`
@@ -254,8 +279,9 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     int cur_u = -1, stage = 0;
     uint32_t kphase = 0, qphase = 0;
     bool ok = true;
-    for (int item = item0; item < item1 && ok; ++item) {
-        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+    ItemTc it = {};
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
         if (it.u != cur_u) {
             ok = mbar_wait(&tl.q_empty, qphase ^ 1, &tl.abort_flag);
             if (!ok) break;
@@ -303,8 +329,9 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
     uint32_t kphase = 0, qphase = 0, aphase[2] = {0, 0};
     bool ok = true;
     int prev_u = -1;
-    for (int item = item0; item < item1 && ok; ++item) {
-        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+    ItemTc it = {};
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
         if (it.u != cur_u) {
             if (prev_u >= 0) umma_commit(&tl.q_empty);     // every MMA on the previous unit's Q has been issued
             ok = mbar_wait(&tl.q_full, qphase, &tl.abort_flag);
@@ -421,8 +448,9 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             zsum[job] = 0.f;
         }
     };
-    for (int item = item0; item < item1 && ok; ++item) {
-        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, a.p.num_kv_heads, item);
+    ItemTc it = {};
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
         if (it.u != cur_u) {
             if (cur_u >= 0) flush(cur_u);
             cur_u = it.u;
@@ -534,8 +562,9 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     int cur_u = -1, buf = 0, par = 0;
     uint32_t aphase[2] = {0, 0}, ephase = 0;
     bool ok = true;
-    for (int item = item0; item < item1 && ok; ++item) {
-        const ItemTc it = decode_item_tc(tl.seq, a.seq_start, a.seq_len, a.p.num_seqs, Hkv, item);
+    ItemTc it = {};
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
         if (it.u != cur_u) {
             if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
             // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
@@ -624,6 +653,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         tl.abort_flag = 0;
         fence_barrier_init();
     }
+    for (int t = threadIdx.x; t < a.p.num_seqs; t += kThreadsTc) tl.start[t] = a.seq_start[t];
     build_seq_tables(tl.seq, a.seq_len, a.p.num_seqs);       // ends with __syncthreads()
     if (warp == kEpiWarps + 1) tmem_alloc(&tl.tmem_base, 512);
     tc_fence_before();

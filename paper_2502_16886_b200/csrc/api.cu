@@ -23,7 +23,7 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     size_t off = 0;
     // partials: per (tile, head, row) for the generic path, per (CTA + unit, padded row) for the tensor-core path
     const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
-    const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, 2 * (256 + U) * rows_pad);
+    const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
     w.part_off = off;   w.part_bytes = align256((size_t)part_items * sizeof(float2));                      off += w.part_bytes;
     w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
     w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 8) * sizeof(int32_t));                         off += w.cnt_bytes;

@@ -426,10 +426,6 @@ __device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
     return m;
 }
 
-// The two epilogue warpgroups each own one accumulator buffer and take alternate
-// jobs (job counter parity = buffer = warpgroup).  The two warps that share an SM
-// sub-partition are therefore out of phase: while one waits for its next
-// accumulator, the other keeps the exponential pipe busy.
 __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1)
 {
     const TcShape &sh = a.sh;
@@ -437,27 +433,20 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int wg = warp >> 2, lane_base = (warp & 3) * 32;
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
-    int cur_u = -1;
-    uint32_t jc = 0, phase = 0;                 // job counter (all jobs), phase of this warpgroup's buffer
-    // running reference and sum of this thread's rows: [job of the tile][row block of the job]
-    float cref[2][2], zsum[2][2];
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) { cref[j][h] = -INFINITY; zsum[j][h] = 0.f; }
+    int cur_u = -1, buf = 0;
+    uint32_t aphase[2] = {0, 0};
+    // per job slot (row block 2*job + wg): running reference and sum of this thread's row
+    float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
     bool ok = true;
     auto flush = [&](int u) {
-        // one partial per (CTA, unit, warpgroup); rows this warpgroup never saw carry (-inf, 0)
-        float2 *dst = a.part + (int64_t)(2 * (blockIdx.x + u) + wg) * sh.Rpad;
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int rb = 2 * j + h, row = rb * kTile + lane_base + lane;
-                if (j < sh.jobs1 && rb < sh.rblocks && row < sh.R) dst[row] = make_float2(cref[j][h], zsum[j][h]);
-                cref[j][h] = -INFINITY;
-                zsum[j][h] = 0.f;
-            }
+        for (int job = 0; job < sh.jobs1; ++job) {
+            const int rb = 2 * job + wg;
+            const int row = rb * kTile + lane_base + lane;
+            if (rb < sh.rblocks && row < sh.R)
+                a.part[(int64_t)(blockIdx.x + u) * sh.Rpad + row] = make_float2(cref[job], zsum[job]);
+            cref[job] = -INFINITY;
+            zsum[job] = 0.f;
+        }
     };
     ItemTc it = {};
     if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
@@ -466,74 +455,68 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (cur_u >= 0) flush(cur_u);
             cur_u = it.u;
         }
-#pragma unroll
-        for (int job = 0; job < 2; ++job) {
-            if (job >= sh.jobs1 || !ok) continue;
-            const bool mine = (int)(jc & 1u) == wg;
-            ++jc;
-            if (!mine) continue;
-            ok = mbar_wait(&tl.acc_full[wg], phase, &tl.abort_flag);
-            if (!ok) continue;
-            phase ^= 1;
+        for (int job = 0; job < sh.jobs1 && ok; ++job) {
+            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
+            if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int rb = 2 * job + h;
-                if (rb >= sh.rblocks) continue;
+            const int rb = 2 * job + wg;
+            if (rb < sh.rblocks) {
                 const int row = rb * kTile + lane_base + lane;
                 const int pos = it.n - w + (row % w);               // position of this row's query
                 int limit = pos - it.tile_start + 1;                // visible positions of the tile: [0, limit)
                 limit = (row < sh.R) ? max(0, min(kTile, limit)) : 0;
-                const uint32_t taddr = tmem_base + (uint32_t)wg * 256u + (uint32_t)h * 128u + ((uint32_t)lane_base << 16);
+                const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)wg * 128u + ((uint32_t)lane_base << 16);
                 const bool full = __all_sync(0xffffffffu, limit == kTile);
-                bool need_max = (cref[job][h] == -INFINITY) && limit > 0;
+                bool need_max = (cref[job] == -INFINITY) && limit > 0;
                 float zt = 0.f;
                 for (int attempt = 0; attempt < 2; ++attempt) {
                     if (__any_sync(0xffffffffu, need_max)) {
                         const float m = row_max_tile(taddr, scale, limit);
-                        if (need_max && m > cref[job][h]) {
-                            zsum[job][h] = (cref[job][h] == -INFINITY) ? 0.f : zsum[job][h] * ex2(cref[job][h] - m);
-                            cref[job][h] = m;
+                        if (need_max && m > cref[job]) {
+                            zsum[job] = (cref[job] == -INFINITY) ? 0.f : zsum[job] * ex2(cref[job] - m);
+                            cref[job] = m;
                         }
                     }
-                    zt = full ? row_sum_tile<false>(taddr, scale, cref[job][h], limit)
-                              : row_sum_tile<true>(taddr, scale, cref[job][h], limit);
+                    zt = full ? row_sum_tile<false>(taddr, scale, cref[job], limit)
+                              : row_sum_tile<true>(taddr, scale, cref[job], limit);
                     need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
                     if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
                 }
-                if (limit > 0) zsum[job][h] += zt;
+                if (limit > 0) zsum[job] += zt;
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[wg]);
+            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
+            aphase[buf] ^= 1;
+            buf ^= 1;
         }
     }
     if (cur_u >= 0 && ok) flush(cur_u);
 }
 
 // Pass 2: thread = position.  Sum over the rows that see it of 2^(y - L[row]).
-// One accumulator: ncol columns (a multiple of 16, at most 256) taken in chunks
-// of 32 (the last may be 16), next chunk in flight.
+// One accumulator's share of a warpgroup: ncol_wg columns (a multiple of 16, at most
+// 128) taken in chunks of 32 (the last may be 16), next chunk in flight.
 template <bool MASKED>
-__device__ inline float col_sum_job(uint32_t taddr, float scale, const float *lse, int rbase, int ncol,
+__device__ inline float col_sum_job(uint32_t taddr, float scale, const float *lse, int rbase, int ncol_wg,
                                     int w, int pos_gap)
 {
     // pos_gap = i - (n - w): row r sees position i iff (r mod w) >= pos_gap
     uint32_t ra[32] = {}, rb[32] = {};
     float s0 = 0.f, s1 = 0.f;
-    if (ncol >= 32) tmem_ld32_issue(taddr, ra); else tmem_ld16_issue(taddr, ra);
+    if (ncol_wg >= 32) tmem_ld32_issue(taddr, ra); else tmem_ld16_issue(taddr, ra);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        if (c * 32 < ncol) {
+    for (int c = 0; c < 4; ++c) {
+        if (c * 32 < ncol_wg) {
             uint32_t (&cur)[32] = (c & 1) ? rb : ra;
             uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
             tmem_ld_wait(cur);
-            if (c + 1 < 8 && (c + 1) * 32 < ncol) {
-                if (ncol - (c + 1) * 32 >= 32) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
+            if (c + 1 < 4 && (c + 1) * 32 < ncol_wg) {
+                if (ncol_wg - (c + 1) * 32 >= 32) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
                 else tmem_ld16_issue(taddr + (c + 1) * 32, nxt);
             }
             const int r0 = rbase + c * 32;
-            const int width = min(32, ncol - c * 32);
+            const int width = min(32, ncol_wg - c * 32);
             int rloc = MASKED ? r0 % w : 0;
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
@@ -575,28 +558,27 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int tid = threadIdx.x;                                   // 0..255
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
-    int cur_u = -1, par = 0;
-    uint32_t jc = 0, phase = 0, ephase = 0;
+    const int ncol_wg = sh.ncol / 2;                               // columns per warpgroup (multiple of 16)
+    int cur_u = -1, buf = 0, par = 0;
+    uint32_t aphase[2] = {0, 0}, ephase = 0;
     bool ok = true;
-    const int pos_in_tile = lane_base + lane;
     ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, Hkv, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, Hkv)) {
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
         if (it.u != cur_u) {
             if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
             // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
-            // left per (CTA, unit, warpgroup), in ascending order (the same in every CTA that needs it)
+            // left per (CTA, unit), in ascending CTA order (the same order in every CTA that needs it)
             const int ts = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
             const int ib = tl.seq.tiles[it.s] * Hkv + it.g * ts;
-            const int s_lo = 2 * (cta_of_item(ib, items, ctas) + it.u);
-            const int s_hi = 2 * (cta_of_item(ib + ts - 1, items, ctas) + it.u) + 1;
+            const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
             for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
                 float M = -INFINITY, Z = 0.f;
-                for (int c0 = s_lo; c0 <= s_hi; c0 += 8) {
+                for (int c0 = c_lo; c0 <= c_hi; c0 += 8) {
                     float2 pr[8];                                  // eight independent loads in flight
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
-                        pr[q] = (c0 + q <= s_hi) ? __ldcg(&a.part[(int64_t)(c0 + q) * sh.Rpad + r])
+                        pr[q] = (c0 + q <= c_hi) ? __ldcg(&a.part[(int64_t)(c0 + q + it.u) * sh.Rpad + r])
                                                  : make_float2(-INFINITY, 0.f);
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -611,49 +593,37 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!(ok = epi_sync(tl, ephase))) break;
             cur_u = it.u;
         }
+        const int pos_in_tile = lane_base + lane;
         const int i = it.tile_start + pos_in_tile;
         const int pos_gap = i - (it.n - w);
         // tile wholly before the window and wholly inside the sequence: every row sees every position
         const bool full = it.tile_start + kTile <= it.n - w + 1;
-        const int cnt = max(1, min(min(w, it.n), it.n - i));
-        const float norm = 1.f / ((float)cnt * (float)G);
-        float *dst = a.scores + (int64_t)it.g * a.total_tokens + it.pack + i;
-#pragma unroll
-        for (int job = 0; job < 2; ++job) {
-            if (job >= sh.nb || !ok) continue;
-            const bool mine = (int)(jc & 1u) == wg;
-            ++jc;
-            if (!mine) continue;
-            ok = mbar_wait(&tl.acc_full[wg], phase, &tl.abort_flag);
-            if (!ok) continue;
-            phase ^= 1;
+        float acc = 0.f;
+        for (int job = 0; job < sh.nb && ok; ++job) {
+            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (uint32_t)wg * 256u + ((uint32_t)lane_base << 16);
-            const float acc = full ? col_sum_job<false>(taddr, scale, tl.lse, job * sh.ncol, sh.ncol, w, pos_gap)
-                                   : col_sum_job<true>(taddr, scale, tl.lse, job * sh.ncol, sh.ncol, w, pos_gap);
+            const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)(wg * ncol_wg) + ((uint32_t)lane_base << 16);
+            const int rbase = job * sh.ncol + wg * ncol_wg;
+            acc += full ? col_sum_job<false>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap)
+                        : col_sum_job<true>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[wg]);
-            if (sh.nb == 1) {
-                if (i < it.n) {
-                    const float sc = acc * norm;
-                    if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
-                    *dst = sc;
-                }
-            } else {
-                tl.stage[par][job][pos_in_tile] = acc;     // two accumulators per tile: the halves meet in shared memory
-            }
+            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
+            aphase[buf] ^= 1;
+            buf ^= 1;
         }
         if (!ok) break;
-        if (sh.nb == 2) {
-            if (!(ok = epi_sync(tl, ephase))) break;
-            if (wg == 0 && i < it.n) {
-                const float sc = (tl.stage[par][0][pos_in_tile] + tl.stage[par][1][pos_in_tile]) * norm;
-                if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
-                *dst = sc;
-            }
-            par ^= 1;     // the other staging buffer is free: its readers passed this item's barrier
+        tl.stage[par][wg][pos_in_tile] = acc;
+        if (!(ok = epi_sync(tl, ephase))) break;
+        if (wg == 0 && i < it.n) {
+            const float tot = tl.stage[par][0][pos_in_tile] + tl.stage[par][1][pos_in_tile];
+            const int cnt = min(min(w, it.n), it.n - i);
+            const float sc = tot / (float)cnt / (float)G;
+            if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
+            a.scores[(int64_t)it.g * a.total_tokens + it.pack + i] = sc;
         }
+        par ^= 1;     // the other staging buffer is free: its readers passed this item's barrier
     }
 }
 
@@ -678,7 +648,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         for (int s = 0; s < 4; ++s) { mbar_init(&tl.k_full[s], 1); mbar_init(&tl.k_empty[s], 1); }
         mbar_init(&tl.q_full, 1);
         mbar_init(&tl.q_empty, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps); }
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();

@@ -120,20 +120,27 @@ struct MinOp { __device__ int operator()(int a, int b) const { return min(a, b);
 struct MaxOpU { __device__ uint32_t operator()(uint32_t a, uint32_t b) const { return max(a, b); } };
 struct AddOpF { __device__ float operator()(float a, float b) const { return a + b; } };
 
-// Ranks [0, count) in the order given by `pos_of` are split into one contiguous
-// segment per warp; inside a segment the lanes interleave, so every load is a
-// coalesced 128-byte line.  seg_totals leaves the exclusive prefix of the warp
-// sums in wpre[0..kWarps) and the grand total in wpre[kWarps].
-__device__ inline int seg_len(int count) { return ceil_div(ceil_div(count, kWarps), 32) * 32; }
+// Ranks [lo, lo + len) in the order given by `pos_of` are split into one
+// contiguous segment per warp; inside a segment the lanes interleave, so every
+// load is a coalesced 128-byte line, and eight loads are in flight per thread.
+// range_totals leaves the exclusive prefix of the warp sums in wpre[0..kWarps)
+// and the total in wpre[kWarps].
+__device__ inline int seg_len(int len) { return ceil_div(ceil_div(len, kWarps), 32) * 32; }
 
 template <typename PosOf>
-__device__ inline u64 seg_totals(const UnitView &v, int count, PosOf pos_of, u64 *wpre)
+__device__ inline u64 range_totals(const UnitView &v, int lo, int len, PosOf pos_of, u64 *wpre)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int seg = seg_len(count);
-    const int w0 = min(count, warp * seg), w1 = min(count, w0 + seg);
+    const int seg = seg_len(len);
+    const int w0 = lo + min(len, warp * seg), w1 = lo + min(len, (warp + 1) * seg);
     u64 local = 0;
-    for (int j = w0 + lane; j < w1; j += 32) local += sq_at(v, pos_of(v, j));
+    for (int j = w0 + lane; j < w1; j += 32 * 8) {
+        u64 x[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) x[q] = (j + 32 * q < w1) ? sq_at(v, pos_of(v, j + 32 * q)) : 0ull;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) local += x[q];
+    }
     for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
     __syncthreads();
     if (lane == 0) wpre[warp] = local;
@@ -149,31 +156,38 @@ __device__ inline u64 seg_totals(const UnitView &v, int count, PosOf pos_of, u64
 }
 
 // First rank count j (1-based) with C_j >= c_min, or INT_MAX, given the warp
-// prefixes of seg_totals: the first warp whose segment end reaches c_min holds
-// the crossing and resolves it 32 ranks at a time.
+// prefixes that range_totals left for ranks [0, count).  The segment whose end
+// first reaches c_min holds the crossing; it is split over the warps again until
+// it is 32 ranks long, which one warp resolves with a scan and a ballot.
 template <typename PosOf>
-__device__ inline int seg_find(const UnitView &v, int count, PosOf pos_of, u64 c_min, const u64 *wpre, int *ibuf)
+__device__ inline int range_find(const UnitView &v, int count, PosOf pos_of, u64 c_min, u64 *wpre, int *ibuf)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int seg = seg_len(count);
-    const int w0 = min(count, warp * seg), w1 = min(count, w0 + seg);
-    const u64 end = warp + 1 < kWarps ? wpre[warp + 1] : wpre[kWarps];
-    const bool first_hit = w1 > w0 && end >= c_min && wpre[warp] < c_min;   // prefixes are monotone: at most one warp
-    __syncthreads();
-    if (threadIdx.x == 0) ibuf[0] = INT_MAX;
-    __syncthreads();
-    if (first_hit) {
-        u64 run = wpre[warp];
-        int found = w1;
-        for (int base = w0; base < w1; base += 32) {
-            const int j = base + lane;
-            u64 x = j < w1 ? sq_at(v, pos_of(v, j)) : 0ull;
-            x = warp_incl_scan(x);
-            const unsigned m = __ballot_sync(0xffffffffu, j < w1 && run + x >= c_min);
-            if (m) { found = base + __ffs(m); break; }
-            run += __shfl_sync(0xffffffffu, x, 31);
+    const int lane = threadIdx.x & 31;
+    int lo = 0, len = count;
+    u64 base = 0;
+    for (;;) {
+        // every thread reads the same prefixes and finds the same segment
+        const int seg = seg_len(len);
+        int hit = -1;
+        for (int wv = 0; wv < kWarps; ++wv) {
+            const u64 end = base + wpre[wv + 1 < kWarps ? wv + 1 : kWarps];
+            if (min(len, wv * seg) < min(len, (wv + 1) * seg) && end >= c_min) { hit = wv; break; }
         }
-        if (lane == 0) ibuf[0] = found;
+        if (hit < 0) return INT_MAX;
+        const int nlo = lo + min(len, hit * seg), nlen = lo + min(len, (hit + 1) * seg) - nlo;
+        base += wpre[hit];
+        lo = nlo;
+        len = nlen;
+        if (len <= 32) break;
+        range_totals(v, lo, len, pos_of, wpre);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int j = lo + lane;
+        u64 x = lane < len ? sq_at(v, pos_of(v, j)) : 0ull;
+        x = warp_incl_scan(x);
+        const unsigned m = __ballot_sync(0xffffffffu, lane < len && base + x >= c_min);
+        if (lane == 0) ibuf[0] = m ? lo + __ffs(m) : lo + len;
     }
     __syncthreads();
     const int found = ibuf[0];
@@ -188,6 +202,8 @@ struct SelectSmem {
     float fbuf[kWarps + 1];
     unsigned int hcnt[256];
     u64 hsum[256];
+    unsigned int wcnt[kWarps][257];   // per-warp private histograms (padded: one bank per warp for a digit)
+    u64 wsum[kWarps][257];
     int pack;
     u64 c_min;
     // radix state
@@ -202,9 +218,13 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
     uint32_t mx = 0;
     bool bad = false;
     for (int h = 0; h < v.heads; ++h)
-        for (int i = threadIdx.x; i < v.n; i += kThreads) {
-            const uint32_t b = mag_bits(v.sc[(int64_t)h * v.head_stride + i]);
-            if ((b >> 23) == 255u) bad = true; else mx = max(mx, b);
+        for (int i = threadIdx.x; i < v.n; i += kThreads * 8) {
+            uint32_t b[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                b[q] = (i + q * kThreads < v.n) ? mag_bits(v.sc[(int64_t)h * v.head_stride + i + q * kThreads]) : 0u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { if ((b[q] >> 23) == 255u) bad = true; else mx = max(mx, b[q]); }
         }
     if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
     mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
@@ -214,10 +234,16 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
     const float f = ldexpf(1.0f, 127 - emax);
     float acc = 0.f;
     for (int h = 0; h < v.heads; ++h)
-        for (int i = threadIdx.x; i < v.n; i += kThreads) {
-            const uint32_t b = mag_bits(v.sc[(int64_t)h * v.head_stride + i]);
-            const float a = ((b >> 23) == 255u) ? 0.f : __uint_as_float(b) * f;
-            acc = fmaf(a, a, acc);
+        for (int i = threadIdx.x; i < v.n; i += kThreads * 8) {
+            uint32_t b[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                b[q] = (i + q * kThreads < v.n) ? mag_bits(v.sc[(int64_t)h * v.head_stride + i + q * kThreads]) : 0u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float a = ((b[q] >> 23) == 255u) ? 0.f : __uint_as_float(b[q]) * f;
+                acc = fmaf(a, a, acc);
+            }
         }
     acc = block_reduce<float>(acc, sm.fbuf, AddOpF());
     // C_n = acc * 2^(2 (emax - 127)); put C_n * 2^S in [2^60, 2^61)
@@ -240,7 +266,8 @@ __global__ void __launch_bounds__(kThreads)
 select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_len,
                      int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status)
 {
-    __shared__ SelectSmem sm;
+    extern __shared__ __align__(16) unsigned char select_smem_raw[];
+    SelectSmem &sm = *reinterpret_cast<SelectSmem *>(select_smem_raw);
     const int Hkv = p.num_kv_heads;
     const bool layer = p.scope == REFREE_SCOPE_LAYER;
     const int s = layer ? blockIdx.x : blockIdx.x / Hkv;
@@ -269,10 +296,10 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
         cut.sbias = v.sbias;
         if (p.rank_mode == REFREE_RANK_POSITION) {
             // one pass in rank order gives C_n and the warp prefixes the search needs
-            const u64 Cn = seg_totals(v, n, PosRank(), sm.wpre);
+            const u64 Cn = range_totals(v, 0, n, PosRank(), sm.wpre);
             if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
             __syncthreads();
-            const int j = seg_find(v, n, PosRank(), sm.c_min, sm.wpre, sm.ibuf);
+            const int j = range_find(v, n, PosRank(), sm.c_min, sm.wpre, sm.ibuf);
             cut.b = max(j == INT_MAX ? n : j, floor_b);
         } else {
             // score ranking: when the protected prefix covers the sequence the order is 0..n-1
@@ -281,13 +308,13 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
             u64 Cn;
             {   // C_n over every position (the order does not matter for an integer sum)
                 UnitView all = v; all.lead = n; all.w_eff = 0;
-                Cn = seg_totals(all, n, ProtRank(), sm.wpre);
+                Cn = range_totals(all, 0, n, ProtRank(), sm.wpre);
             }
             if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
             __syncthreads();
             const u64 c_min = sm.c_min;
-            const u64 Sprot = seg_totals(v, prot, ProtRank(), sm.wpre);
-            const int jp = seg_find(v, prot, ProtRank(), c_min, sm.wpre, sm.ibuf);
+            const u64 Sprot = range_totals(v, 0, prot, ProtRank(), sm.wpre);
+            const int jp = range_find(v, prot, ProtRank(), c_min, sm.wpre, sm.ibuf);
             int jstar = n;
             cut.prot_kept = prot;
             cut.tau = 0ull;                       // keep every unprotected position ...
@@ -301,16 +328,40 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
                 bool any = true;
                 for (int level = 0; level < levels && any; ++level) {
                     const int shift = 56 - 8 * level;
-                    for (int t = threadIdx.x; t < 256; t += kThreads) { sm.hcnt[t] = 0u; sm.hsum[t] = 0ull; }
+                    // each warp fills a histogram of its own (no contention between warps on a
+                    // popular digit); thread t then adds up digit t over the warps
+                    const int warp = threadIdx.x >> 5;
+                    for (int t = threadIdx.x; t < kWarps * 257; t += kThreads) {
+                        (&sm.wcnt[0][0])[t] = 0u;
+                        (&sm.wsum[0][0])[t] = 0ull;
+                    }
                     __syncthreads();
                     const u64 prefix = sm.prefix;
-                    for (int i = v.lead + threadIdx.x; i < n - v.w_eff; i += kThreads) {
-                        const u64 key = key_at(v, i);
-                        if (level == 0 || (key >> (shift + 8)) == prefix) {
-                            const int dgt = (int)((key >> shift) & 255ull);
-                            atomicAdd(&sm.hcnt[dgt], 1u);
-                            atomicAdd(&sm.hsum[dgt], v.heads == 1 ? sq_at(v, i) : key);
+                    for (int i0 = v.lead + threadIdx.x; i0 < n - v.w_eff; i0 += kThreads * 4) {
+                        u64 key[4], val[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int i = i0 + q * kThreads;
+                            const bool in = i < n - v.w_eff;
+                            key[q] = in ? key_at(v, i) : 0ull;
+                            val[q] = !in ? 0ull : (v.heads == 1 ? sq_fixed((uint32_t)(key[q] >> 32), v.sbias) : key[q]);
                         }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (i0 + q * kThreads < n - v.w_eff && (level == 0 || (key[q] >> (shift + 8)) == prefix)) {
+                                const int dgt = (int)((key[q] >> shift) & 255ull);
+                                atomicAdd(&sm.wcnt[warp][dgt], 1u);
+                                atomicAdd(&sm.wsum[warp][dgt], val[q]);
+                            }
+                        }
+                    }
+                    __syncthreads();
+                    if (threadIdx.x < 256) {
+                        unsigned int c = 0u;
+                        u64 sumv = 0ull;
+                        for (int wv = 0; wv < kWarps; ++wv) { c += sm.wcnt[wv][threadIdx.x]; sumv += sm.wsum[wv][threadIdx.x]; }
+                        sm.hcnt[threadIdx.x] = c;
+                        sm.hsum[threadIdx.x] = sumv;
                     }
                     __syncthreads();
                     // inclusive sums from the top digit down; thread t owns digit 255 - t
@@ -450,7 +501,16 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     Cut *cuts = reinterpret_cast<Cut *>(ws + lay.cut_off);
     const int U = p.num_seqs * p.num_kv_heads;
     const int sel_units = p.scope == REFREE_SCOPE_LAYER ? p.num_seqs : U;
-    select_budget_kernel<<<sel_units, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(select_budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)sizeof(SelectSmem));
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    select_budget_kernel<<<sel_units, kThreads, sizeof(SelectSmem), st>>>(p, scores, seq_len, total_tokens, lengths,
+                                                                            cuts, dev_status);
     if (!emit) {               // the caller forms the offsets itself and needs no index list
         count_launches(1);
         return cudaGetLastError();

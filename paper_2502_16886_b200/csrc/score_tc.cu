@@ -176,19 +176,20 @@ __host__ __device__ inline uint32_t make_idesc(int n)
 struct TcShape {
     int R;        // query rows per unit: G * window
     int Rpad;     // rows of the shared-memory Q image (multiple of 128)
-    int rblocks;  // 128-row blocks (pass 1 A operands)
-    int jobs1;    // pass-1 accumulators per tile (two row blocks each)
-    int nb;       // pass-2 accumulators per tile
-    int ncol;     // pass-2 columns (rows of Q) per accumulator: R / nb
+    int rblocks;  // 128-row blocks: pass-1 accumulators per tile (A operands)
+    int cblocks;  // pass-2 accumulators per tile
+    int ncol;     // pass-2 columns (rows of Q) per accumulator: R / cblocks, at most 128
     int stages;   // K tile ring depth
     int rank4;    // K tensor map has a sequence axis
 };
 
 struct TcSmemTail {
-    uint64_t k_full[4], k_empty[4], q_full, q_empty, acc_full[2], acc_empty[2], epi_bar;
+    uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
+    uint64_t acc_full[4], acc_empty[4];       // accumulator (warpgroup * 2 + slot): 128 tensor-memory columns each
+    uint64_t half_ready[3];                   // pass 2: warpgroup 1 has staged its half of a tile
     uint32_t tmem_base;
     int abort_flag;
-    alignas(16) float stage[2][2][kTile];     // pass 2: per item parity, per warpgroup partial column sums
+    alignas(16) float stage[3][kTile];        // pass 2: warpgroup 1's partial column sums, three tiles deep
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
     SeqTables seq;
     int32_t start[kMaxSeqs];                  // copy of seq_start
@@ -317,6 +318,11 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     }
 }
 
+// Accumulators: four of 128 tensor-memory columns.  Block b of a tile (a 128-row
+// block of Q in pass 1, a block of `ncol` rows of Q in pass 2) goes to warpgroup
+// b & 1, which owns two accumulators and alternates between them, so the MMA of a
+// warpgroup's next block runs while it reads the current one, and the two
+// warpgroups (hence the two warps sharing an SM sub-partition) drift out of phase.
 template <int PASS>
 __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
                                 uint32_t tmem_base, int item0, int item1)
@@ -325,8 +331,9 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
     const uint32_t q_lo = desc_lo(smem_u32(smem_q)), k_lo = desc_lo(smem_u32(smem_k));
     const uint32_t q_half = (uint32_t)(sh.Rpad * 128) >> 4;      // distance between the two 64-column halves of Q
     const uint32_t idesc1 = make_idesc(kTile), idesc2 = make_idesc(sh.ncol);
-    int cur_u = -1, stage = 0, buf = 0;
-    uint32_t kphase = 0, qphase = 0, aphase[2] = {0, 0};
+    const int blocks = PASS == 1 ? sh.rblocks : sh.cblocks;
+    int cur_u = -1, stage = 0;
+    uint32_t kphase = 0, qphase = 0, cnt0 = 0, cnt1 = 0;         // blocks issued to each warpgroup
     bool ok = true;
     int prev_u = -1;
     ItemTc it = {};
@@ -344,35 +351,31 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
         if (!ok) break;
         tc_fence_after();
         const uint32_t kt_lo = k_lo + (uint32_t)stage * (kTileBytes >> 4);
-        const int jobs = PASS == 1 ? sh.jobs1 : sh.nb;
-        for (int job = 0; job < jobs && ok; ++job) {
-            ok = mbar_wait(&tl.acc_empty[buf], aphase[buf] ^ 1, &tl.abort_flag);
+        for (int b = 0; b < blocks && ok; ++b) {
+            const int wg = b & 1;
+            const uint32_t cnt = wg ? cnt1 : cnt0;
+            const int acc = wg * 2 + (int)(cnt & 1u);
+            ok = mbar_wait(&tl.acc_empty[acc], ((cnt >> 1) & 1u) ^ 1u, &tl.abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d0 = tmem_base + (uint32_t)buf * 256u;
+            const uint32_t d0 = tmem_base + (uint32_t)acc * 128u;
             if (PASS == 1) {
-                for (int half_acc = 0; half_acc < 2; ++half_acc) {
-                    const int rb = 2 * job + half_acc;
-                    if (rb >= sh.rblocks) break;
-                    const uint32_t qa = q_lo + (uint32_t)rb * (kHalfBytes >> 4);
+                const uint32_t qa = q_lo + (uint32_t)b * (kHalfBytes >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t h = kk >> 2, ko = (kk & 3) * 2;          // 32 bytes per K step of 16
-                        umma_bf16(d0 + half_acc * 128, qa + h * q_half + ko, kt_lo + h * (kHalfBytes >> 4) + ko,
-                                  kDescHi, idesc1, kk > 0);
-                    }
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t h = kk >> 2, ko = (kk & 3) * 2;          // 32 bytes per K step of 16
+                    umma_bf16(d0, qa + h * q_half + ko, kt_lo + h * (kHalfBytes >> 4) + ko, kDescHi, idesc1, kk > 0);
                 }
             } else {
-                const uint32_t qb = q_lo + (uint32_t)job * (uint32_t)(sh.ncol * 128 >> 4);
+                const uint32_t qb = q_lo + (uint32_t)b * (uint32_t)(sh.ncol * 128 >> 4);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t h = kk >> 2, ko = (kk & 3) * 2;
                     umma_bf16(d0, kt_lo + h * (kHalfBytes >> 4) + ko, qb + h * q_half + ko, kDescHi, idesc2, kk > 0);
                 }
             }
-            umma_commit(&tl.acc_full[buf]);
-            aphase[buf] ^= 1;
-            buf ^= 1;
+            umma_commit(&tl.acc_full[acc]);
+            if (wg) ++cnt1; else ++cnt0;
         }
         umma_commit(&tl.k_empty[stage]);
         if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
@@ -433,19 +436,20 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int wg = warp >> 2, lane_base = (warp & 3) * 32;
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
-    int cur_u = -1, buf = 0;
-    uint32_t aphase[2] = {0, 0};
-    // per job slot (row block 2*job + wg): running reference and sum of this thread's row
+    int cur_u = -1;
+    uint32_t cnt = 0;                            // blocks this warpgroup has consumed
+    // running reference and sum of this thread's rows: row blocks wg and wg + 2
     float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
     bool ok = true;
     auto flush = [&](int u) {
-        for (int job = 0; job < sh.jobs1; ++job) {
-            const int rb = 2 * job + wg;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int rb = wg + 2 * j;
             const int row = rb * kTile + lane_base + lane;
             if (rb < sh.rblocks && row < sh.R)
-                a.part[(int64_t)(blockIdx.x + u) * sh.Rpad + row] = make_float2(cref[job], zsum[job]);
-            cref[job] = -INFINITY;
-            zsum[job] = 0.f;
+                a.part[(int64_t)(blockIdx.x + u) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
+            cref[j] = -INFINITY;
+            zsum[j] = 0.f;
         }
     };
     ItemTc it = {};
@@ -455,40 +459,40 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (cur_u >= 0) flush(cur_u);
             cur_u = it.u;
         }
-        for (int job = 0; job < sh.jobs1 && ok; ++job) {
-            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
-            if (!ok) break;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int rb = wg + 2 * j;
+            if (rb >= sh.rblocks || !ok) continue;
+            const int acc = wg * 2 + (int)(cnt & 1u);
+            ok = mbar_wait(&tl.acc_full[acc], (cnt >> 1) & 1u, &tl.abort_flag);
+            if (!ok) continue;
+            ++cnt;
             tc_fence_after();
-            const int rb = 2 * job + wg;
-            if (rb < sh.rblocks) {
-                const int row = rb * kTile + lane_base + lane;
-                const int pos = it.n - w + (row % w);               // position of this row's query
-                int limit = pos - it.tile_start + 1;                // visible positions of the tile: [0, limit)
-                limit = (row < sh.R) ? max(0, min(kTile, limit)) : 0;
-                const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)wg * 128u + ((uint32_t)lane_base << 16);
-                const bool full = __all_sync(0xffffffffu, limit == kTile);
-                bool need_max = (cref[job] == -INFINITY) && limit > 0;
-                float zt = 0.f;
-                for (int attempt = 0; attempt < 2; ++attempt) {
-                    if (__any_sync(0xffffffffu, need_max)) {
-                        const float m = row_max_tile(taddr, scale, limit);
-                        if (need_max && m > cref[job]) {
-                            zsum[job] = (cref[job] == -INFINITY) ? 0.f : zsum[job] * ex2(cref[job] - m);
-                            cref[job] = m;
-                        }
+            const int row = rb * kTile + lane_base + lane;
+            const int pos = it.n - w + (row % w);               // position of this row's query
+            int limit = pos - it.tile_start + 1;                // visible positions of the tile: [0, limit)
+            limit = (row < sh.R) ? max(0, min(kTile, limit)) : 0;
+            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
+            const bool full = __all_sync(0xffffffffu, limit == kTile);
+            bool need_max = (cref[j] == -INFINITY) && limit > 0;
+            float zt = 0.f;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                if (__any_sync(0xffffffffu, need_max)) {
+                    const float m = row_max_tile(taddr, scale, limit);
+                    if (need_max && m > cref[j]) {
+                        zsum[j] = (cref[j] == -INFINITY) ? 0.f : zsum[j] * ex2(cref[j] - m);
+                        cref[j] = m;
                     }
-                    zt = full ? row_sum_tile<false>(taddr, scale, cref[job], limit)
-                              : row_sum_tile<true>(taddr, scale, cref[job], limit);
-                    need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
-                    if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
                 }
-                if (limit > 0) zsum[job] += zt;
+                zt = full ? row_sum_tile<false>(taddr, scale, cref[j], limit)
+                          : row_sum_tile<true>(taddr, scale, cref[j], limit);
+                need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
+                if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
             }
+            if (limit > 0) zsum[j] += zt;
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
-            aphase[buf] ^= 1;
-            buf ^= 1;
+            if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
         }
     }
     if (cur_u >= 0 && ok) flush(cur_u);
@@ -558,13 +562,33 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int tid = threadIdx.x;                                   // 0..255
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
-    const int ncol_wg = sh.ncol / 2;                               // columns per warpgroup (multiple of 16)
-    int cur_u = -1, buf = 0, par = 0;
-    uint32_t aphase[2] = {0, 0}, ephase = 0;
-    bool ok = true;
+    const int pos_in_tile = lane_base + lane;
+    const bool two_halves = sh.cblocks > 1;                        // both warpgroups contribute to a tile
+    int cur_u = -1;
+    uint32_t cnt = 0, ephase = 0, tcount = 0;                      // blocks consumed, tiles seen
+    // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
+    float pend_acc = 0.f, pend_norm = 0.f;
+    float *pend_dst = nullptr;
+    uint32_t pend_tile = 0;
+    bool pending = false, ok = true;
+    auto finish_pending = [&]() -> bool {
+        if (!pending) return true;
+        float tot = pend_acc;
+        if (two_halves) {
+            if (!mbar_wait(&tl.half_ready[pend_tile % 3u], (pend_tile / 3u) & 1u, &tl.abort_flag)) return false;
+            tot += tl.stage[pend_tile % 3u][pos_in_tile];
+        }
+        if (pend_dst) {
+            const float sc = tot * pend_norm;
+            if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
+            *pend_dst = sc;
+        }
+        pending = false;
+        return true;
+    };
     ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
+    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, Hkv, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, Hkv)) {
         if (it.u != cur_u) {
             if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
             // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
@@ -593,38 +617,46 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!(ok = epi_sync(tl, ephase))) break;
             cur_u = it.u;
         }
-        const int pos_in_tile = lane_base + lane;
+        // the previous tile is completed before any accumulator of this tile is handed back, which
+        // keeps warpgroup 1 at most two tiles ahead of the staging slot being read here
+        if (wg == 0 && !(ok = finish_pending())) break;
         const int i = it.tile_start + pos_in_tile;
         const int pos_gap = i - (it.n - w);
         // tile wholly before the window and wholly inside the sequence: every row sees every position
         const bool full = it.tile_start + kTile <= it.n - w + 1;
-        float acc = 0.f;
-        for (int job = 0; job < sh.nb && ok; ++job) {
-            ok = mbar_wait(&tl.acc_full[buf], aphase[buf], &tl.abort_flag);
-            if (!ok) break;
+        float accv = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int cb = wg + 2 * j;
+            if (cb >= sh.cblocks || !ok) continue;
+            const int acc = wg * 2 + (int)(cnt & 1u);
+            ok = mbar_wait(&tl.acc_full[acc], (cnt >> 1) & 1u, &tl.abort_flag);
+            if (!ok) continue;
+            ++cnt;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)(wg * ncol_wg) + ((uint32_t)lane_base << 16);
-            const int rbase = job * sh.ncol + wg * ncol_wg;
-            acc += full ? col_sum_job<false>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap)
-                        : col_sum_job<true>(taddr, scale, tl.lse, rbase, ncol_wg, w, pos_gap);
+            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
+            accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap)
+                         : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[buf]);
-            aphase[buf] ^= 1;
-            buf ^= 1;
+            if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
         }
         if (!ok) break;
-        tl.stage[par][wg][pos_in_tile] = acc;
-        if (!(ok = epi_sync(tl, ephase))) break;
-        if (wg == 0 && i < it.n) {
-            const float tot = tl.stage[par][0][pos_in_tile] + tl.stage[par][1][pos_in_tile];
-            const int cnt = min(min(w, it.n), it.n - i);
-            const float sc = tot / (float)cnt / (float)G;
-            if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
-            a.scores[(int64_t)it.g * a.total_tokens + it.pack + i] = sc;
+        if (wg == 0) {
+            const int cnt_i = max(1, min(min(w, it.n), it.n - i));
+            pend_acc = accv;
+            pend_norm = 1.f / ((float)cnt_i * (float)G);
+            pend_dst = i < it.n ? a.scores + (int64_t)it.g * a.total_tokens + it.pack + i : nullptr;
+            pend_tile = tcount;
+            pending = true;
+        } else if (two_halves) {
+            tl.stage[tcount % 3u][pos_in_tile] = accv;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tl.half_ready[tcount % 3u]);
         }
-        par ^= 1;     // the other staging buffer is free: its readers passed this item's barrier
+        ++tcount;
     }
+    if (wg == 0 && ok) finish_pending();
 }
 
 // ---------------------------------------------------------------- kernels ----
@@ -648,7 +680,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         for (int s = 0; s < 4; ++s) { mbar_init(&tl.k_full[s], 1); mbar_init(&tl.k_empty[s], 1); }
         mbar_init(&tl.q_full, 1);
         mbar_init(&tl.q_empty, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps); }
+        for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
+        for (int b = 0; b < 3; ++b) mbar_init(&tl.half_ready[b], kEpiWarps / 2);
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();
@@ -712,12 +745,11 @@ bool shape_for(const refree_params &p, TcShape &sh)
     const int64_t R = (int64_t)G * p.window;
     if (R < 32 || R > kMaxRowsTc) return false;
     sh.R = (int)R;
-    sh.nb = (sh.R + 255) / 256;
-    if (sh.R % (32 * sh.nb) != 0) return false;           // each warpgroup takes ncol/2 columns in chunks of 16
-    sh.ncol = sh.R / sh.nb;
+    sh.cblocks = (sh.R + kTile - 1) / kTile;
+    if (sh.R % (16 * sh.cblocks) != 0) return false;      // accumulators are read in chunks of 16 columns
+    sh.ncol = sh.R / sh.cblocks;
     sh.rblocks = (sh.R + kTile - 1) / kTile;
     sh.Rpad = sh.rblocks * kTile;
-    sh.jobs1 = (sh.rblocks + 1) / 2;
     sh.stages = sh.Rpad <= 256 ? 4 : 2;
     sh.rank4 = p.k_stride_seq != 0;
     return true;

@@ -187,6 +187,7 @@ struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
     uint64_t acc_full[4], acc_empty[4];       // accumulator (warpgroup * 2 + slot): 128 tensor-memory columns each
     uint64_t half_ready[3];                   // pass 2: warpgroup 1 has staged its half of a tile
+    uint64_t turn[2];                         // ping-pong of the exponential phase between the warpgroups
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) float stage[3][kTile];        // pass 2: warpgroup 1's partial column sums, three tiles deep
@@ -267,6 +268,23 @@ __device__ inline bool epi_sync(TcSmemTail &tl, uint32_t &phase)
     const bool ok = mbar_wait(&tl.epi_bar, phase, &tl.abort_flag);
     phase ^= 1;
     return ok;
+}
+
+// Ping-pong of the exponential phase.  The exponentials saturate the special
+// function pipe when one warp per SM sub-partition runs them, so the two
+// warpgroups take turns (warpgroup 0's block k, warpgroup 1's block k, ...): the
+// barrier waits, the index arithmetic and the hand-back of an accumulator by one
+// warpgroup are hidden behind the exponentials of the other.  Used when both
+// warpgroups get the same number of blocks per tile.
+__device__ inline bool turn_begin(TcSmemTail &tl, int wg, uint32_t k)
+{
+    // warpgroup 0 waits for warpgroup 1's block k - 1 (nothing before its first), warpgroup 1 for warpgroup 0's block k
+    return mbar_wait(&tl.turn[wg], wg == 0 ? ((k & 1u) ^ 1u) : (k & 1u), &tl.abort_flag);
+}
+__device__ inline void turn_end(TcSmemTail &tl, int wg)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(&tl.turn[wg ^ 1]);
 }
 
 // --------------------------------------------------------- producer / MMA -----
@@ -440,6 +458,15 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
     uint32_t cnt = 0;                            // blocks this warpgroup has consumed
     // running reference and sum of this thread's rows: row blocks wg and wg + 2
     float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
+    int rmod[2];
+    bool rvalid[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int row = (wg + 2 * j) * kTile + lane_base + lane;
+        rmod[j] = row % w;                       // offset of the row's query inside the window
+        rvalid[j] = row < sh.R;
+    }
+    const bool pingpong = (sh.rblocks & 1) == 0;
     bool ok = true;
     auto flush = [&](int u) {
 #pragma unroll
@@ -468,14 +495,19 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!ok) continue;
             ++cnt;
             tc_fence_after();
-            const int row = rb * kTile + lane_base + lane;
-            const int pos = it.n - w + (row % w);               // position of this row's query
-            int limit = pos - it.tile_start + 1;                // visible positions of the tile: [0, limit)
-            limit = (row < sh.R) ? max(0, min(kTile, limit)) : 0;
+            int limit = kTile;                                  // visible positions of the tile: [0, limit)
+            const bool full = it.tile_start + kTile <= it.n - w + 1;   // tile wholly before the window
+            if (!full) {
+                limit = it.n - w + rmod[j] - it.tile_start + 1;     // up to this row's own position
+                limit = (rvalid[j]) ? max(0, min(kTile, limit)) : 0;
+            } else if (!rvalid[j]) {
+                limit = 0;
+            }
+            const bool uniform = __all_sync(0xffffffffu, limit == kTile);
             const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
-            const bool full = __all_sync(0xffffffffu, limit == kTile);
             bool need_max = (cref[j] == -INFINITY) && limit > 0;
             float zt = 0.f;
+            if (pingpong && !(ok = turn_begin(tl, wg, cnt - 1u))) continue;
             for (int attempt = 0; attempt < 2; ++attempt) {
                 if (__any_sync(0xffffffffu, need_max)) {
                     const float m = row_max_tile(taddr, scale, limit);
@@ -484,11 +516,12 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
                         cref[j] = m;
                     }
                 }
-                zt = full ? row_sum_tile<false>(taddr, scale, cref[j], limit)
-                          : row_sum_tile<true>(taddr, scale, cref[j], limit);
+                zt = uniform ? row_sum_tile<false>(taddr, scale, cref[j], limit)
+                             : row_sum_tile<true>(taddr, scale, cref[j], limit);
                 need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
                 if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
             }
+            if (pingpong) turn_end(tl, wg);
             if (limit > 0) zsum[j] += zt;
             tc_fence_before();
             __syncwarp();
@@ -564,6 +597,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
     const int pos_in_tile = lane_base + lane;
     const bool two_halves = sh.cblocks > 1;                        // both warpgroups contribute to a tile
+    const bool pingpong = (sh.cblocks & 1) == 0;
     int cur_u = -1;
     uint32_t cnt = 0, ephase = 0, tcount = 0;                      // blocks consumed, tiles seen
     // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
@@ -635,8 +669,10 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             ++cnt;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
+            if (pingpong && !(ok = turn_begin(tl, wg, cnt - 1u))) continue;
             accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap)
                          : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap);
+            if (pingpong) turn_end(tl, wg);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
@@ -682,6 +718,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
         for (int b = 0; b < 3; ++b) mbar_init(&tl.half_ready[b], kEpiWarps / 2);
+        for (int b = 0; b < 2; ++b) mbar_init(&tl.turn[b], kEpiWarps / 2);
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();

@@ -187,7 +187,6 @@ struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
     uint64_t acc_full[4], acc_empty[4];       // accumulator (warpgroup * 2 + slot): 128 tensor-memory columns each
     uint64_t half_ready[3];                   // pass 2: warpgroup 1 has staged its half of a tile
-    uint64_t turn[2];                         // ping-pong of the exponential phase between the warpgroups
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) float stage[3][kTile];        // pass 2: warpgroup 1's partial column sums, three tiles deep
@@ -268,23 +267,6 @@ __device__ inline bool epi_sync(TcSmemTail &tl, uint32_t &phase)
     const bool ok = mbar_wait(&tl.epi_bar, phase, &tl.abort_flag);
     phase ^= 1;
     return ok;
-}
-
-// Ping-pong of the exponential phase.  The exponentials saturate the special
-// function pipe when one warp per SM sub-partition runs them, so the two
-// warpgroups take turns (warpgroup 0's block k, warpgroup 1's block k, ...): the
-// barrier waits, the index arithmetic and the hand-back of an accumulator by one
-// warpgroup are hidden behind the exponentials of the other.  Used when both
-// warpgroups get the same number of blocks per tile.
-__device__ inline bool turn_begin(TcSmemTail &tl, int wg, uint32_t k)
-{
-    // warpgroup 0 waits for warpgroup 1's block k - 1 (nothing before its first), warpgroup 1 for warpgroup 0's block k
-    return mbar_wait(&tl.turn[wg], wg == 0 ? ((k & 1u) ^ 1u) : (k & 1u), &tl.abort_flag);
-}
-__device__ inline void turn_end(TcSmemTail &tl, int wg)
-{
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) mbar_arrive(&tl.turn[wg ^ 1]);
 }
 
 // --------------------------------------------------------- producer / MMA -----
@@ -466,7 +448,6 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
         rmod[j] = row % w;                       // offset of the row's query inside the window
         rvalid[j] = row < sh.R;
     }
-    const bool pingpong = (sh.rblocks & 1) == 0;
     bool ok = true;
     auto flush = [&](int u) {
 #pragma unroll
@@ -507,7 +488,6 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
             bool need_max = (cref[j] == -INFINITY) && limit > 0;
             float zt = 0.f;
-            if (pingpong && !(ok = turn_begin(tl, wg, cnt - 1u))) continue;
             for (int attempt = 0; attempt < 2; ++attempt) {
                 if (__any_sync(0xffffffffu, need_max)) {
                     const float m = row_max_tile(taddr, scale, limit);
@@ -521,7 +501,6 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
                 need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
                 if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
             }
-            if (pingpong) turn_end(tl, wg);
             if (limit > 0) zsum[j] += zt;
             tc_fence_before();
             __syncwarp();
@@ -597,7 +576,6 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
     const int pos_in_tile = lane_base + lane;
     const bool two_halves = sh.cblocks > 1;                        // both warpgroups contribute to a tile
-    const bool pingpong = (sh.cblocks & 1) == 0;
     int cur_u = -1;
     uint32_t cnt = 0, ephase = 0, tcount = 0;                      // blocks consumed, tiles seen
     // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
@@ -669,10 +647,8 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             ++cnt;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
-            if (pingpong && !(ok = turn_begin(tl, wg, cnt - 1u))) continue;
             accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap)
                          : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap);
-            if (pingpong) turn_end(tl, wg);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
@@ -718,7 +694,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
         for (int b = 0; b < 3; ++b) mbar_init(&tl.half_ready[b], kEpiWarps / 2);
-        for (int b = 0; b < 2; ++b) mbar_init(&tl.turn[b], kEpiWarps / 2);
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();

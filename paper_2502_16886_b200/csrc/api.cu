@@ -26,7 +26,7 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
     w.part_off = off;   w.part_bytes = align256((size_t)part_items * sizeof(float2));                      off += w.part_bytes;
     w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
-    w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
+    w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 256 + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
     w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
     w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
     w.kept_off = off;   w.kept_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(int32_t)); off += w.kept_bytes;

@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 
 #include "refree_internal.cuh"
@@ -253,6 +254,8 @@ struct TcArgs {
     TcShape sh;
     const int32_t *seq_start, *seq_len;
     float2 *part;        // [ctas + units][Rpad]
+    uint32_t *flags;     // fused launch: flags[c] == epoch once CTA c has written its pass-1 partials
+    uint32_t epoch;
     float *scores;
     int64_t total_tokens;
     int32_t *dev_status;
@@ -269,16 +272,22 @@ __device__ inline bool epi_sync(TcSmemTail &tl, uint32_t &phase)
     return ok;
 }
 
+// Loop state that survives from pass 1 to pass 2 when both run in one launch.
+struct RingState { int stage = 0; uint32_t kphase = 0, qphase = 0; };
+struct MmaState : RingState { uint32_t cnt0 = 0, cnt1 = 0; int prev_u = -1; };
+struct EpiState { uint32_t cnt = 0, ephase = 0; };
+
 // --------------------------------------------------------- producer / MMA -----
 template <int PASS>
 __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, const CUtensorMap *mapk,
                                      unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
-                                     int item0, int item1)
+                                     int item0, int item1, RingState &rs)
 {
     const TcShape &sh = a.sh;
     const int G = a.p.num_q_heads / a.p.num_kv_heads;
-    int cur_u = -1, stage = 0;
-    uint32_t kphase = 0, qphase = 0;
+    int cur_u = -1;
+    int &stage = rs.stage;
+    uint32_t &kphase = rs.kphase, &qphase = rs.qphase;
     bool ok = true;
     ItemTc it = {};
     if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
@@ -325,17 +334,17 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
 // warpgroups (hence the two warps sharing an SM sub-partition) drift out of phase.
 template <int PASS>
 __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
-                                uint32_t tmem_base, int item0, int item1)
+                                uint32_t tmem_base, int item0, int item1, MmaState &ms)
 {
     const TcShape &sh = a.sh;
     const uint32_t q_lo = desc_lo(smem_u32(smem_q)), k_lo = desc_lo(smem_u32(smem_k));
     const uint32_t q_half = (uint32_t)(sh.Rpad * 128) >> 4;      // distance between the two 64-column halves of Q
     const uint32_t idesc1 = make_idesc(kTile), idesc2 = make_idesc(sh.ncol);
     const int blocks = PASS == 1 ? sh.rblocks : sh.cblocks;
-    int cur_u = -1, stage = 0;
-    uint32_t kphase = 0, qphase = 0, cnt0 = 0, cnt1 = 0;         // blocks issued to each warpgroup
+    int cur_u = -1;
+    int &stage = ms.stage, &prev_u = ms.prev_u;
+    uint32_t &kphase = ms.kphase, &qphase = ms.qphase, &cnt0 = ms.cnt0, &cnt1 = ms.cnt1;   // blocks issued per warpgroup
     bool ok = true;
-    int prev_u = -1;
     ItemTc it = {};
     if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
     for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
@@ -429,7 +438,8 @@ __device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
     return m;
 }
 
-__device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1)
+__device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1,
+                                      EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -437,7 +447,7 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
     int cur_u = -1;
-    uint32_t cnt = 0;                            // blocks this warpgroup has consumed
+    uint32_t &cnt = es.cnt;                      // blocks this warpgroup has consumed
     // running reference and sum of this thread's rows: row blocks wg and wg + 2
     float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
     int rmod[2];
@@ -566,7 +576,7 @@ __device__ inline int cta_of_item(int x, int items, int ctas)
 }
 
 __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1,
-                                      int items, int ctas)
+                                      int items, int ctas, EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -577,7 +587,8 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     const int pos_in_tile = lane_base + lane;
     const bool two_halves = sh.cblocks > 1;                        // both warpgroups contribute to a tile
     int cur_u = -1;
-    uint32_t cnt = 0, ephase = 0, tcount = 0;                      // blocks consumed, tiles seen
+    uint32_t &cnt = es.cnt, &ephase = es.ephase;                   // blocks consumed, phase of the epilogue barrier
+    uint32_t tcount = 0;                                           // tiles seen
     // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
     float pend_acc = 0.f, pend_norm = 0.f;
     float *pend_dst = nullptr;
@@ -608,6 +619,22 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             const int ts = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
             const int ib = tl.seq.tiles[it.s] * Hkv + it.g * ts;
             const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
+            if (a.flags) {
+                // one launch for both passes: the partials of this unit come from CTAs that may still be in
+                // pass 1; wait (bounded) until each of them has published
+                for (int c = c_lo + tid; c <= c_hi; c += kEpiWarps * 32) {
+                    bool seen = false;
+                    for (uint32_t spin = 0; spin < kSpinLimit && !seen; ++spin) {
+                        uint32_t v;
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.flags + c) : "memory");
+                        seen = v == a.epoch;
+                        if (!seen) { if (tl.abort_flag) break; __nanosleep(spin > 64 ? 256 : 32); }
+                    }
+                    if (!seen) tl.abort_flag = 1;
+                }
+                if (!(ok = epi_sync(tl, ephase))) break;
+                if (tl.abort_flag) { ok = false; break; }
+            }
             for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
                 float M = -INFINITY, Z = 0.f;
                 for (int c0 = c_lo; c0 <= c_hi; c0 += 8) {
@@ -713,13 +740,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     const int item0 = active ? range_begin(blockIdx.x, items, ctas) : 0;
     const int item1 = active ? range_begin(blockIdx.x + 1, items, ctas) : 0;
 
+    // PASS 1 or 2: that pass alone; PASS 3: both passes in this launch (all CTAs co-resident)
     if (warp < kEpiWarps) {
-        if (PASS == 1) epilogue_pass1(a, tl, tmem_base, item0, item1);
-        else epilogue_pass2(a, tl, tmem_base, item0, item1, items, ctas);
+        EpiState es;
+        if (PASS != 2) epilogue_pass1(a, tl, tmem_base, item0, item1, es);
+        if (PASS == 3) {
+            // publish: this CTA's partials are in memory
+            __threadfence();
+            epi_sync(tl, es.ephase);
+            if (threadIdx.x == 0)
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(a.epoch) : "memory");
+        }
+        if (PASS != 1) epilogue_pass2(a, tl, tmem_base, item0, item1, items, ctas, es);
     } else if (warp == kEpiWarps) {
-        if (lane == 0) producer_loop<PASS>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1);
+        if (lane == 0) {
+            RingState rs;
+            if (PASS != 2) producer_loop<1>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1, rs);
+            if (PASS != 1) producer_loop<2>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1, rs);
+        }
     } else {
-        if (lane == 0) mma_loop<PASS>(a, smem_q, smem_k, tl, tmem_base, item0, item1);
+        if (lane == 0) {
+            MmaState ms;
+            if (PASS != 2) mma_loop<1>(a, smem_q, smem_k, tl, tmem_base, item0, item1, ms);
+            if (PASS != 1) mma_loop<2>(a, smem_q, smem_k, tl, tmem_base, item0, item1, ms);
+        }
     }
     __syncwarp();
     // Common exit.  In the normal case the epilogue has consumed every accumulator,
@@ -812,6 +856,7 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
             return cudaErrorInvalidValue;
     }
     static int sm_count[64] = {};
+    static bool coop_ok[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -824,6 +869,11 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e != cudaSuccess) return e;
+        int coop = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) coop = 0;
+        coop_ok[dev] = coop != 0;
         sm_count[dev] = std::min(n, kMaxCtas);
     }
     const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
@@ -839,6 +889,27 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.dev_status = dev_status;
     const size_t smem = smem_bytes(sh);
     if (smem > 232448) return cudaErrorInvalidValue;
+    a.flags = nullptr;
+    a.epoch = 0;
+    if (coop_ok[dev]) {
+        // Both passes in one cooperative launch (co-residency of all CTAs is what makes the wait of pass 2
+        // on other CTAs' pass 1 safe).  The flags hold a per-call token, so a workspace left over from an
+        // earlier call needs no clearing.
+        static std::atomic<uint32_t> token{0x5eed1234u};
+        uint32_t epoch = token.fetch_add(1u, std::memory_order_relaxed) + 1u;
+        if (epoch == 0u) epoch = token.fetch_add(1u, std::memory_order_relaxed) + 1u;
+        a.flags = reinterpret_cast<uint32_t *>(ws + lay.cnt_off);
+        a.epoch = epoch;
+        void *args[3] = {(void *)&mapq, (void *)&mapk, (void *)&a};
+        const cudaError_t ce = cudaLaunchCooperativeKernel((const void *)score_tc_kernel<3>, dim3(ctas), dim3(kThreadsTc),
+                                                           args, smem, st);
+        if (ce == cudaSuccess) {
+            count_launches(1);
+            return cudaGetLastError();
+        }
+        (void)cudaGetLastError();        // not launchable as one grid here: fall back to one launch per pass
+        a.flags = nullptr;
+    }
     score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
     score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
     count_launches(2);

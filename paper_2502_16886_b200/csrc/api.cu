@@ -26,6 +26,7 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
     w.part_off = off;   w.part_bytes = align256((size_t)part_items * sizeof(float2));                      off += w.part_bytes;
     w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
+    w.grp_off = off;    w.grp_bytes = align256((size_t)(tiles * p.num_kv_heads * 4) * sizeof(GroupPartial));  off += w.grp_bytes;
     w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 256 + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
     w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
     w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
@@ -72,13 +73,18 @@ static refree_status check_kv_layout(const refree_params *p, const void *k, cons
 
 static refree_status from_cuda(cudaError_t e) { return e == cudaSuccess ? REFREE_OK : REFREE_ERR_CUDA; }
 
+static bool use_tc(const refree_params &p, const void *q_win)
+{
+    return score_tc_supported(p) && !(reinterpret_cast<uintptr_t>(q_win) & 15);
+}
+
 static cudaError_t run_score(const refree_params &p, const void *q_win, const void *k,
                              const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
                              float *scores, char *ws, const Workspace &lay, int32_t *dev_status,
-                             cudaStream_t st)
+                             cudaStream_t st, GroupPartial *groups = nullptr)
 {
-    if (score_tc_supported(p) && !(reinterpret_cast<uintptr_t>(q_win) & 15))
-        return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
+    if (use_tc(p, q_win))
+        return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st, groups);
     return launch_score_generic(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
 }
 
@@ -212,13 +218,19 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
     int32_t *kept = kept_idx ? kept_idx : (ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off));
     cudaError_t e = cudaSuccess;
     // a frozen layer needs no scores unless the caller asked for them
+    // position ranking per head on the tensor-core path: the scoring kernel also leaves the per-32-position
+    // sums of squares, and the stopping rule reads those instead of every score
+    GroupPartial *groups = nullptr;
+    if (use_tc(*p, q_win) && p->rank_mode == REFREE_RANK_POSITION && p->scope == REFREE_SCOPE_HEAD && !p->force_full &&
+        total_tokens > 0)
+        groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
     if (total_tokens > 0 && (!p->force_full || scores))
-        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs);
+        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);
     if (e != cudaSuccess) return REFREE_ERR_CUDA;
     // with two-range kept sets and no index list wanted, the compaction kernel forms the offsets itself
     const bool lean = ranges && !kept;
     e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs,
-                      !lean);
+                      !lean, groups);
     if (e != cudaSuccess) return REFREE_ERR_CUDA;
     e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, lean ? offsets : nullptr, k_out,
                        v_out, capacity_rows, device_status, cs);

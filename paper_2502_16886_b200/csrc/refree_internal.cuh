@@ -19,7 +19,8 @@ constexpr uint32_t kSpinLimit = 1u << 22;
 // Layout of the caller-provided workspace.  All offsets are multiples of 256.
 struct Workspace {
     size_t part_off, part_bytes;       // per (tile, head, row) softmax partials (float2: max, sum)
-    size_t lse_off, lse_bytes;         // per (unit, row) log2-sum-exp of the row's logits
+    size_t lse_off, lse_bytes;         // generic path: per (unit, row) log2-sum-exp of the row's logits
+    size_t grp_off, grp_bytes;         // per 32 positions: exact partial sum of squared scores (GroupPartial)
     size_t cnt_off, cnt_bytes;         // per unit arrival counters (zeroed by each call)
     size_t cut_off, cut_bytes;         // per unit selection result (struct Cut)
     size_t scores_off, scores_bytes;   // scratch scores when the caller passes none
@@ -40,6 +41,19 @@ struct Cut {
     int32_t prot_kept;  // score ranking: protected positions kept
     int32_t sbias;      // fixed-point exponent bias of the unit's squares (see select.cu)
 };
+
+// Sum of squared scores of 32 consecutive positions of one unit, written by the
+// scoring kernel so that the stopping rule need not re-read every score.
+//   max_bits  bit pattern of the largest score of the group (0 when all are zero)
+//   sum       sum over the group of floor(a^2 * 2^(308 - 2E)), E = exponent field of
+//             max_bits (at least 1): exact integer squares, at most 2^61 in total
+// Records of unit (s, g) are contiguous: index (tiles[s] * Hkv + g * tiles_of(s)) * 4 + i / 32.
+struct GroupPartial {
+    uint32_t max_bits;
+    uint32_t pad;
+    unsigned long long sum;
+};
+constexpr int kGroupShift = 8;   // the squared mantissa (below 2^48) of the group's largest score lands below 2^56
 
 Workspace workspace_layout(const refree_params &p, int64_t total_tokens);
 
@@ -84,6 +98,22 @@ __device__ inline int find_seq(const int32_t *table, int B, int x)
     return lo;
 }
 
+// |a| as an integer: non-negative floats order like their bit patterns
+__device__ inline uint32_t mag_bits(float a) { return __float_as_uint(a) & 0x7fffffffu; }
+
+// floor(a^2 * 2^S) from the bits of |a|, where 2 * exponent_field + sbias is the left
+// shift of the exact 48-bit squared mantissa (S = sbias + 300); non-finite values count as zero
+__device__ inline unsigned long long sq_fixed(uint32_t bits, int sbias)
+{
+    const uint32_t e = bits >> 23;
+    if (e == 255u) return 0ull;
+    const uint32_t m = (bits & 0x7fffffu) | (e ? 0x800000u : 0u);
+    const unsigned long long mm = (unsigned long long)m * m;     // exact, below 2^48
+    const int sh = 2 * (int)(e ? e : 1u) + sbias;
+    if (sh >= 0) return sh < 16 ? mm << sh : ~0ull >> 2;
+    return -sh < 48 ? mm >> -sh : 0ull;
+}
+
 template <typename T> __device__ inline float to_float(T v);
 template <> __device__ inline float to_float<float>(float v) { return v; }
 template <> __device__ inline float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -99,12 +129,13 @@ bool score_tc_supported(const refree_params &p);
 cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
                             const int32_t *seq_start, const int32_t *seq_len,
                             int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
-                            int32_t *dev_status, cudaStream_t st);
+                            int32_t *dev_status, cudaStream_t st, GroupPartial *groups = nullptr);
 
 cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
                           int64_t total_tokens, int32_t *lengths, int64_t *offsets,
                           int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,
-                          int32_t *dev_status, cudaStream_t st, bool emit = true);
+                          int32_t *dev_status, cudaStream_t st, bool emit = true,
+                          const GroupPartial *groups = nullptr);
 
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            const int32_t *seq_start, const int32_t *seq_len,

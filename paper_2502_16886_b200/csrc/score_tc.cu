@@ -254,6 +254,7 @@ struct TcArgs {
     TcShape sh;
     const int32_t *seq_start, *seq_len;
     float2 *part;        // [ctas + units][Rpad]
+    GroupPartial *groups; // nullable: per 32 positions, exact sum of squared scores for the stopping rule
     uint32_t *flags;     // fused launch: flags[c] == epoch once CTA c has written its pass-1 partials
     uint32_t epoch;
     float *scores;
@@ -592,6 +593,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
     float pend_acc = 0.f, pend_norm = 0.f;
     float *pend_dst = nullptr;
+    GroupPartial *pend_grp = nullptr;
     uint32_t pend_tile = 0;
     bool pending = false, ok = true;
     auto finish_pending = [&]() -> bool {
@@ -601,10 +603,19 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!mbar_wait(&tl.half_ready[pend_tile % 3u], (pend_tile / 3u) & 1u, &tl.abort_flag)) return false;
             tot += tl.stage[pend_tile % 3u][pos_in_tile];
         }
+        float sc = 0.f;
         if (pend_dst) {
-            const float sc = tot * pend_norm;
+            sc = tot * pend_norm;
             if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
             *pend_dst = sc;
+        }
+        if (pend_grp) {
+            // this warp's 32 positions: largest score, and the exact squares summed at a scale set by it
+            const uint32_t bits = (pend_dst && isfinite(sc)) ? mag_bits(sc) : 0u;
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, bits);
+            unsigned long long sq = sq_fixed(bits, kGroupShift - 2 * max(1, (int)(mx >> 23)));
+            for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            if (lane == 0) { GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq; *pend_grp = gp; }
         }
         pending = false;
         return true;
@@ -686,6 +697,9 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             pend_acc = accv;
             pend_norm = 1.f / ((float)cnt_i * (float)G);
             pend_dst = i < it.n ? a.scores + (int64_t)it.g * a.total_tokens + it.pack + i : nullptr;
+            pend_grp = a.groups ? a.groups + ((int64_t)tl.seq.tiles[it.s] * Hkv + (int64_t)it.g * it.ntiles + it.tile) * 4 +
+                                      (warp & 3)
+                                : nullptr;
             pend_tile = tcount;
             pending = true;
         } else if (two_halves) {
@@ -829,7 +843,7 @@ bool score_tc_supported(const refree_params &p)
 cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
                             const int32_t *seq_start, const int32_t *seq_len,
                             int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
-                            int32_t *dev_status, cudaStream_t st)
+                            int32_t *dev_status, cudaStream_t st, GroupPartial *groups)
 {
     TcShape sh;
     if (!shape_for(p, sh)) return cudaErrorInvalidValue;
@@ -884,6 +898,7 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.seq_start = seq_start;
     a.seq_len = seq_len;
     a.part = reinterpret_cast<float2 *>(ws + lay.part_off);
+    a.groups = groups;
     a.scores = scores;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;

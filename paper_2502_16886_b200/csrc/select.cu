@@ -41,20 +41,6 @@ struct UnitView {
     int sbias;              // fixed point: a^2 * 2^S = mantissa^2 * 2^(2 * exponent_field + sbias)
 };
 
-__device__ inline uint32_t mag_bits(float a) { return __float_as_uint(a) & 0x7fffffffu; }
-
-// floor(a^2 * 2^S) from the bits of |a|; non-finite values count as zero
-__device__ inline u64 sq_fixed(uint32_t bits, int sbias)
-{
-    const uint32_t e = bits >> 23;
-    if (e == 255u) return 0ull;
-    const uint32_t m = (bits & 0x7fffffu) | (e ? 0x800000u : 0u);
-    const u64 mm = (u64)m * m;                                   // exact, below 2^48
-    const int sh = 2 * (int)(e ? e : 1u) + sbias;
-    if (sh >= 0) return sh < 16 ? mm << sh : ~0ull >> 2;
-    return -sh < 48 ? mm >> -sh : 0ull;
-}
-
 __device__ inline u64 sq_at(const UnitView &v, int i)
 {
     u64 acc = 0;
@@ -412,6 +398,126 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     }
 }
 
+// Position ranking, one budget per (sequence, KV head), from the per-32-position
+// partials that the scoring kernel left (GroupPartial): the stopping rule then
+// touches one record per 32 scores plus the 32 scores of the group in which the
+// cumulative sum crosses.  Same rule and fixed point as select_budget_kernel, with
+// each group's sum first brought to the unit's common scale (a right shift).
+__global__ void __launch_bounds__(kThreads)
+select_groups_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_t total_tokens,
+                     const GroupPartial *groups, int32_t *lengths, Cut *cuts)
+{
+    __shared__ u64 ubuf[kWarps + 1];
+    __shared__ int ibuf[kWarps + 1];
+    __shared__ int s_pack, s_tiles;
+    __shared__ u64 s_cmin, s_sink;
+    __shared__ int s_found;
+    const int Hkv = p.num_kv_heads;
+    const int s = blockIdx.x / Hkv, g = blockIdx.x % Hkv;
+    if (threadIdx.x == 0) {
+        int a = 0, b = 0;
+        for (int t = 0; t < s; ++t) { const int nn = max(seq_len[t], 0); a += nn; b += ceil_div(nn, kTile); }
+        s_pack = a;
+        s_tiles = b;
+    }
+    __syncthreads();
+    const int n = max(seq_len[s], 0);
+    const float *sc = scores + (int64_t)g * total_tokens + s_pack;
+    const int lead = min(p.sink, n), w_eff = min(p.window, n);
+    const int floor_b = p.keep_window ? min(n, lead + w_eff) : min(n, 1);
+    const int ng = ceil_div(n, 32);
+    const GroupPartial *gp = groups + ((int64_t)s_tiles * Hkv + (int64_t)g * ceil_div(n, kTile)) * 4;
+    Cut cut;
+    cut.b = n; cut.ties = 0; cut.tau = 0; cut.prot_kept = 0; cut.sbias = 0;
+    if (n > 0) {
+        // common scale: the largest score's squared mantissa below 2^(56 - L), L = log2 of the group count
+        uint32_t mx = 0;
+        for (int k = threadIdx.x; k < ng; k += kThreads) mx = max(mx, gp[k].max_bits);
+        mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(ibuf), MaxOpU());
+        if (mx != 0u) {
+            const int emax = max(1, (int)(mx >> 23));
+            int L = 0;
+            while ((1 << L) < ng) ++L;
+            const int sbias = kGroupShift - 2 * emax - L;
+            cut.sbias = sbias;
+            // mass of the leading positions (ranked first), and of every group without them
+            u64 sink = 0;
+            for (int i = threadIdx.x; i < lead; i += kThreads) sink += sq_fixed(mag_bits(sc[i]), sbias);
+            {
+                u64 tot;
+                block_excl_scan<u64>(sink, ubuf, tot);
+                sink = tot;
+            }
+            auto group_rest = [&](int k) -> u64 {
+                const GroupPartial r = gp[k];
+                const int shift = 2 * (emax - max(1, (int)(r.max_bits >> 23))) + L;
+                u64 v = shift < 64 ? r.sum >> shift : 0ull;
+                if (32 * k < lead) {                   // take the leading positions out of their group
+                    u64 in = 0;
+                    for (int i = 32 * k; i < min(lead, 32 * k + 32); ++i) in += sq_fixed(mag_bits(sc[i]), sbias);
+                    v = v > in ? v - in : 0ull;
+                }
+                return v;
+            };
+            // groups in ranked order: from the last one backwards; thread t owns a contiguous run of them
+            const int per = ceil_div(ng, kThreads);
+            const int r0 = min(ng, (int)threadIdx.x * per), r1 = min(ng, r0 + per);
+            u64 local = 0;
+            for (int r = r0; r < r1; ++r) local += group_rest(ng - 1 - r);
+            u64 rest_total;
+            const u64 before = block_excl_scan<u64>(local, ubuf, rest_total);
+            const u64 Cn = sink + rest_total;
+            if (threadIdx.x == 0) { s_cmin = crossing_level(Cn, (double)p.threshold); s_found = INT_MAX; s_sink = sink; }
+            __syncthreads();
+            const u64 c_min = s_cmin;
+            int jstar = INT_MAX;
+            if (threadIdx.x == 0) {                    // crossing among the leading positions
+                u64 c = 0;
+                for (int i = 0; i < lead; ++i) {
+                    c += sq_fixed(mag_bits(sc[i]), sbias);
+                    if (c >= c_min) { s_found = i + 1; break; }
+                }
+            }
+            __syncthreads();
+            jstar = s_found;
+            __syncthreads();
+            if (jstar == INT_MAX && c_min != ~0ull) {
+                // first group (in ranked order) at whose end the cumulative sum reaches c_min
+                int hit = INT_MAX;
+                u64 run = sink + before, hit_before = 0;
+                for (int r = r0; r < r1; ++r) {
+                    const u64 v = group_rest(ng - 1 - r);
+                    if (run + v >= c_min) { hit = r; hit_before = run; break; }
+                    run += v;
+                }
+                const int first = block_reduce<int>(hit, ibuf, MinOp());
+                if (first != INT_MAX) {
+                    if (hit == first) { ubuf[0] = hit_before; }
+                    __syncthreads();
+                    if (threadIdx.x < 32) {
+                        const int k = ng - 1 - first;
+                        const int hi = min(n, 32 * k + 32) - 1, lo = max(lead, 32 * k);
+                        const int pos = hi - (int)threadIdx.x;
+                        u64 x = pos >= lo ? sq_fixed(mag_bits(sc[pos]), sbias) : 0ull;
+                        x = warp_incl_scan(x);
+                        const unsigned m = __ballot_sync(0xffffffffu, pos >= lo && ubuf[0] + x >= c_min);
+                        // rank count of position pos: the leading ones, then n-1 down to pos
+                        const int last = m ? hi - (__ffs(m) - 1) : lo;
+                        if (threadIdx.x == 0) s_found = lead + (n - last);
+                    }
+                    __syncthreads();
+                    jstar = s_found;
+                }
+            }
+            cut.b = max(jstar == INT_MAX ? n : jstar, floor_b);
+        }
+    }
+    if (threadIdx.x == 0) {
+        lengths[blockIdx.x] = cut.b;
+        cuts[blockIdx.x] = cut;
+    }
+}
+
 // Offsets (running sum of lengths) and the kept positions of each unit, ascending.
 __global__ void __launch_bounds__(kThreads)
 emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_t total_tokens,
@@ -496,7 +602,7 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
 cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
                           int64_t total_tokens, int32_t *lengths, int64_t *offsets,
                           int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,
-                          int32_t *dev_status, cudaStream_t st, bool emit)
+                          int32_t *dev_status, cudaStream_t st, bool emit, const GroupPartial *groups)
 {
     Cut *cuts = reinterpret_cast<Cut *>(ws + lay.cut_off);
     const int U = p.num_seqs * p.num_kv_heads;
@@ -509,8 +615,11 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    select_budget_kernel<<<sel_units, kThreads, sizeof(SelectSmem), st>>>(p, scores, seq_len, total_tokens, lengths,
-                                                                            cuts, dev_status);
+    if (groups && p.rank_mode == REFREE_RANK_POSITION && p.scope == REFREE_SCOPE_HEAD && !p.force_full)
+        select_groups_kernel<<<U, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, groups, lengths, cuts);
+    else
+        select_budget_kernel<<<sel_units, kThreads, sizeof(SelectSmem), st>>>(p, scores, seq_len, total_tokens, lengths,
+                                                                                cuts, dev_status);
     if (!emit) {               // the caller forms the offsets itself and needs no index list
         count_launches(1);
         return cudaGetLastError();

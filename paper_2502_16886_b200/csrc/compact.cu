@@ -11,26 +11,17 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 4;
 
-// L2 policy: rows that are read or written exactly once here (V, and both outputs)
-// are marked evict-first, so that they do not push out the K rows which the scoring
-// kernels have just streamed through L2 and which this kernel reads next.
-__device__ inline uint64_t policy_evict_first()
-{
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ inline int4 ld_stream(const int4 *p, uint64_t pol)
+__device__ inline int4 ld_stream(const int4 *p)
 {
     int4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.s32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-__device__ inline void st_stream(int4 *p, const int4 &v, uint64_t pol)
+__device__ inline void st_stream(int4 *p, const int4 &v)
 {
-    asm volatile("st.global.L2::cache_hint.v4.s32 [%0], {%1,%2,%3,%4}, %5;"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
+    asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -76,7 +67,6 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
     const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
     char *ko = k_out + off * row_bytes, *vo = v_out + off * row_bytes;
     const int32_t *idx = kept_idx ? kept_idx + off : nullptr;
-    const uint64_t pol = policy_evict_first();
     const int64_t nvec = (int64_t)b << vshift;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     for (int64_t e0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; e0 < nvec; e0 += stride * kUnroll) {
@@ -88,15 +78,15 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
                 const int t = (int)(e >> vshift), c = (int)(e & (vec_per_row - 1));
                 const int src = position_ranges ? (t < head ? t : n - b + t) : idx[t];
                 kv[r] = *reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok + c * 16);
-                vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16), pol);
+                vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16));
             }
         }
 #pragma unroll
         for (int r = 0; r < kUnroll; ++r) {
             const int64_t e = e0 + r * stride;
             if (e < nvec) {
-                st_stream(reinterpret_cast<int4 *>(ko + e * 16), kv[r], pol);
-                st_stream(reinterpret_cast<int4 *>(vo + e * 16), vv[r], pol);
+                st_stream(reinterpret_cast<int4 *>(ko + e * 16), kv[r]);
+                st_stream(reinterpret_cast<int4 *>(vo + e * 16), vv[r]);
             }
         }
     }

@@ -89,29 +89,6 @@ __device__ inline void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
 }
-// K tiles of pass 2 are read once more by the compaction kernel: loaded with an
-// evict-last L2 policy (pass 1 and Q use the default).
-__device__ inline uint64_t policy_evict_last()
-{
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ inline void tma_load_3d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
-                                        uint64_t pol)
-{
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-                 "[%0], [%1, {%3, %4, %5}], [%2], %6;"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
-}
-__device__ inline void tma_load_4d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
-                                        int c3, uint64_t pol)
-{
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-                 "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol)
-                 : "memory");
-}
 __device__ inline void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
@@ -312,7 +289,6 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     int cur_u = -1;
     int &stage = rs.stage;
     uint32_t &kphase = rs.kphase, &qphase = rs.qphase;
-    const uint64_t keep = policy_evict_last();
     bool ok = true;
     ItemTc it = {};
     if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
@@ -334,18 +310,10 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
         mbar_expect_tx(&tl.k_full[stage], (uint32_t)kTileBytes);
         unsigned char *dst = smem_k + (size_t)stage * kTileBytes;
         for (int h = 0; h < 2; ++h) {
-            if (PASS == 2) {
-                if (sh.rank4)
-                    tma_load_4d_hint(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g,
-                                     it.s, keep);
-                else
-                    tma_load_3d_hint(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g,
-                                     keep);
-            } else if (sh.rank4) {
+            if (sh.rank4)
                 tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s);
-            } else {
+            else
                 tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g);
-            }
         }
         if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
     }

@@ -486,7 +486,7 @@ select_groups_kernel(refree_params p, const float *scores, const int32_t *seq_le
                 int hit = INT_MAX;
                 u64 run = sink + before, hit_before = 0;
                 for (int r = r0; r < r1; ++r) {
-                    const u64 v = group_rest(ng - 1 - r);
+                    const u64 v = per == 1 ? local : group_rest(ng - 1 - r);   // one group per thread: already in a register
                     if (run + v >= c_min) { hit = r; hit_before = run; break; }
                     run += v;
                 }

@@ -262,26 +262,35 @@ def run_ours(args):
     ms_layer = ms_step / L
     pass_gbs = bytes3 / (ms_layer * 1e-3) / 1e9
 
-    # per-stage device times, one event-bracketed sweep over the layers through the stage entry points
+    # per-stage device times: each stage entry point called back to back over the layers (no synchronisation
+    # inside the bracket, so the GPU never idles waiting for a launch), CUDA events around the sweep
     scores = torch.empty(cfg.num_kv_heads, total, dtype=torch.float32, device=dev)
     kept = torch.empty(cap, dtype=torch.int32, device=dev)
-    stage_ms = {"score": 0.0, "select": 0.0, "compact": 0.0}
-    reps = 3
-    for rep in range(reps + 1):
+    binding.refree_select_budget(params, scores.zero_(), seq_len, total, layers[0]["lengths"], layers[0]["offsets"],
+                                 kept, cap, ws, status)
+    stage_calls = {
+        "score": lambda d: binding.refree_score(params, d["q"], d["k"], seq_start, seq_len, total, scores, ws, status),
+        "select": lambda d: binding.refree_select_budget(params, scores, seq_len, total, d["lengths"], d["offsets"],
+                                                         kept, cap, ws, status),
+        "compact": lambda d: binding.refree_compact(params, d["k"], d["v"], seq_start, seq_len, d["lengths"],
+                                                    d["offsets"], kept, d["k_out"], d["v_out"], cap, status),
+    }
+    stage_ms = {}
+    reps = 5
+    one_layer(layers[-1])                      # leaves real scores behind for the select sweep
+    binding.refree_score(params, layers[-1]["q"], layers[-1]["k"], seq_start, seq_len, total, scores, ws, status)
+    for name, call in stage_calls.items():
         for d in layers:
-            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-            e[0].record()
-            binding.refree_score(params, d["q"], d["k"], seq_start, seq_len, total, scores, ws, status)
-            e[1].record()
-            binding.refree_select_budget(params, scores, seq_len, total, d["lengths"], d["offsets"], kept, cap, ws, status)
-            e[2].record()
-            binding.refree_compact(params, d["k"], d["v"], seq_start, seq_len, d["lengths"], d["offsets"], kept,
-                                   d["k_out"], d["v_out"], cap, status)
-            e[3].record()
-            torch.cuda.synchronize()
-            if rep > 0:
-                for i, name in enumerate(stage_ms):
-                    stage_ms[name] += e[i].elapsed_time(e[i + 1]) / (reps * L)
+            call(d)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for d in layers:
+                call(d)
+        e1.record()
+        torch.cuda.synchronize()
+        stage_ms[name] = e0.elapsed_time(e1) / (reps * L)
     row = cfg.head_dim * cfg.elem_bytes
     kept_rows = rho * cfg.num_kv_heads * total
     stage_bytes = {"score": cfg.num_kv_heads * total * (row + 4), "select": cfg.num_kv_heads * total * 8,

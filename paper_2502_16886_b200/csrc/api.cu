@@ -24,7 +24,9 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     // partials: per (tile, head, row) for the generic path, per (CTA + unit, padded row) for the tensor-core path
     const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
     const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
-    w.part_off = off;   w.part_bytes = align256((size_t)part_items * sizeof(float2));                      off += w.part_bytes;
+    size_t part_bytes = (size_t)part_items * sizeof(float2);
+    if (score_w1_supported(p)) part_bytes = std::max(part_bytes, score_w1_scratch_bytes(p, total_tokens));
+    w.part_off = off;   w.part_bytes = align256(part_bytes);                                               off += w.part_bytes;
     w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
     w.grp_off = off;    w.grp_bytes = align256((size_t)(tiles * p.num_kv_heads * 4) * sizeof(GroupPartial));  off += w.grp_bytes;
     w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 256 + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
@@ -85,6 +87,8 @@ static cudaError_t run_score(const refree_params &p, const void *q_win, const vo
 {
     if (use_tc(p, q_win))
         return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st, groups);
+    if (score_w1_supported(p))
+        return launch_score_w1(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st, groups);
     return launch_score_generic(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st);
 }
 
@@ -221,8 +225,8 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
     // position ranking per head on the tensor-core path: the scoring kernel also leaves the per-32-position
     // sums of squares, and the stopping rule reads those instead of every score
     GroupPartial *groups = nullptr;
-    if (use_tc(*p, q_win) && p->rank_mode == REFREE_RANK_POSITION && p->scope == REFREE_SCOPE_HEAD && !p->force_full &&
-        total_tokens > 0)
+    if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
+        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
         groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
     if (total_tokens > 0 && (!p->force_full || scores))
         e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);

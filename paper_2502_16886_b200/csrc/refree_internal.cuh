@@ -131,6 +131,14 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
                             int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
                             int32_t *dev_status, cudaStream_t st, GroupPartial *groups = nullptr);
 
+// Single query row per head (the paper's default reduced attention): a stream over K on the fp32 pipes.
+bool score_w1_supported(const refree_params &p);
+size_t score_w1_scratch_bytes(const refree_params &p, int64_t total_tokens);
+cudaError_t launch_score_w1(const refree_params &p, const void *q_win, const void *k,
+                            const int32_t *seq_start, const int32_t *seq_len,
+                            int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
+                            int32_t *dev_status, cudaStream_t st, GroupPartial *groups = nullptr);
+
 cudaError_t launch_select(const refree_params &p, const float *scores, const int32_t *seq_len,
                           int64_t total_tokens, int32_t *lengths, int64_t *offsets,
                           int32_t *kept_idx, int64_t capacity_rows, char *ws, const Workspace &lay,

@@ -220,3 +220,15 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert torch.equal(parity.bits(k_out[:rows]), parity.bits(dev_res.k_out[:rows].cpu()))
     assert torch.equal(parity.bits(v_out[:rows]), parity.bits(dev_res.v_out[:rows].cpu()))
     assert torch.equal(scores, dev_res.scores.cpu())
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv", [("bf16", 128, 28, 4), ("fp32", 64, 4, 2), ("bf16", 64, 16, 1), ("fp32", 128, 3, 3)])
+@pytest.mark.parametrize("rank_mode,scope", [(binding.RANK_POSITION, binding.SCOPE_HEAD),
+                                             (binding.RANK_SCORE, binding.SCOPE_HEAD),
+                                             (binding.RANK_POSITION, binding.SCOPE_LAYER)])
+def test_single_query_row_path_shapes_and_modes(dtype, d, hq, hkv, rank_mode, scope):
+    """w = 1 (the paper's default) has a scoring path of its own: group sizes 1..16,
+    both storage types and head dims, ragged lengths down to one token."""
+    cfg = small_cfg(window=1, num_q_heads=hq, num_kv_heads=hkv, dtype=dtype, head_dim=d)
+    lay = workloads.make_layer(cfg, 2, seq_lens=[1, 300, 257, 4000, 31])
+    parity.run_fused_and_check(cfg, lay, rank_mode=rank_mode, scope=scope)

@@ -185,6 +185,9 @@ def run_ours(args):
     build.build()
     binding.lib()
     cfg = workloads.get_config(args.workload)
+    if args.window:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, window=args.window)      # e.g. 1: the paper's default reduced attention
     L = args.layers or cfg.num_layers
     rank_mode = binding.RANK_SCORE if args.rank_mode == "score" else binding.RANK_POSITION
     seq_lens = workloads.sequence_lengths(cfg)
@@ -454,6 +457,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--rank-mode", choices=["position", "score"], default="position")
     ap.add_argument("--layers", type=int, default=0, help="debugging: use fewer layers than the config")
+    ap.add_argument("--window", type=int, default=0, help="override the config's observation window (paper default: 1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -100,95 +100,104 @@ struct W1Args {
     int32_t *dev_status;
 };
 
+// A K row is covered by LPR = row_bytes / 16 lanes, 16 bytes each, so a warp reads
+// 32 / LPR whole rows per load instruction (fully coalesced).  Each lane keeps its
+// slice of the G queries in registers; the partial dot products meet by shuffles.
 template <typename T, int D, int GMAX>
 __global__ void __launch_bounds__(kThreadsW1)
 w1_logits_kernel(W1Args a, const T *q_win, const T *k)
 {
+    constexpr int E = Row16<T>::kElems;              // elements per lane and row
+    constexpr int LPR = D / E;                       // lanes per row: 8, 16 or 32
+    constexpr int RPW = 32 / LPR;                    // rows per warp and load
+    constexpr int kWarpsW1 = kThreadsW1 / 32;
+    constexpr int kRowsPerWarp = kChunk / kWarpsW1;  // 32 positions of the chunk per warp
     __shared__ W1Tables tb;
-    __shared__ __align__(16) float qs[GMAX][D];
-    __shared__ float red[kThreadsW1 / 32][GMAX];
-    __shared__ float bmax[GMAX];
+    __shared__ float2 red[kWarpsW1][GMAX];
     const refree_params &p = a.p;
     const int B = p.num_seqs, Hkv = p.num_kv_heads, G = p.num_q_heads / Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / LPR, part = lane % LPR;   // row of the load this lane helps with, its 16-byte slice
     const float scale = kLog2eW1 * rsqrtf((float)D);
     build_w1_tables(tb, a.seq_len, B);
     const int items = tb.chunks[B] * Hkv;
     int cur_u = -1;
+    float qreg[GMAX][E];
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const W1Item it = decode_w1(tb, B, Hkv, item);
         const int u = it.s * Hkv + it.g;
-        __syncthreads();
-        if (u != cur_u) {                       // the unit's G queries, pre-scaled, as fp32
-            for (int e = threadIdx.x; e < G * D; e += kThreadsW1) {
-                const int hh = e / D, c = e % D;
-                qs[hh][c] = to_float(q_win[((int64_t)it.s * p.num_q_heads + it.g * G + hh) * D + c]) * scale;
-            }
-            cur_u = u;
-            __syncthreads();
-        }
-        const int i = it.pos0 + threadIdx.x;
-        const bool valid = i < it.n;
-        float acc[GMAX];
+        if (u != cur_u) {                            // this lane's slice of the unit's G queries, pre-scaled
 #pragma unroll
-        for (int h = 0; h < GMAX; ++h) acc[h] = 0.f;
-        if (valid) {
-            const char *row = reinterpret_cast<const char *>(
-                k + (int64_t)it.s * p.k_stride_seq + ((int64_t)a.seq_start[it.s] + i) * p.k_stride_tok +
-                (int64_t)it.g * p.k_stride_head);
-            constexpr int E = Row16<T>::kElems;
+            for (int h = 0; h < GMAX; ++h)
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    qreg[h][e] = h < G ? to_float(q_win[((int64_t)it.s * p.num_q_heads + it.g * G + h) * D + part * E + e]) * scale
+                                       : 0.f;
+            cur_u = u;
+        }
+        const char *base = reinterpret_cast<const char *>(
+            k + (int64_t)it.s * p.k_stride_seq + (int64_t)a.seq_start[it.s] * p.k_stride_tok + (int64_t)it.g * p.k_stride_head);
+        const int64_t tok_bytes = p.k_stride_tok * (int64_t)sizeof(T);
+        // running (max, sum) per head over the rows this lane leads
+        float m[GMAX], z[GMAX];
+#pragma unroll
+        for (int h = 0; h < GMAX; ++h) { m[h] = -INFINITY; z[h] = 0.f; }
+        const int wpos0 = it.pos0 + warp * kRowsPerWarp;
 #pragma unroll 4
-            for (int c = 0; c < D / E; ++c) {
-                float kf[8];
-                Row16<T>::load(row + c * 16, kf);
+        for (int r = 0; r < kRowsPerWarp; r += RPW) {
+            const int i = wpos0 + r + sub;
+            const bool valid = i < it.n;
+            float kf[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kf[e] = 0.f;
+            if (valid) Row16<T>::load(base + (int64_t)i * tok_bytes + part * 16, kf);
+            float y[GMAX];
+#pragma unroll
+            for (int h = 0; h < GMAX; ++h) {
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc = fmaf(kf[e], qreg[h][e], acc);
+                y[h] = acc;
+            }
+#pragma unroll
+            for (int o = LPR / 2; o; o >>= 1)
+#pragma unroll
+                for (int h = 0; h < GMAX; ++h)
+                    if (h < G) y[h] += __shfl_xor_sync(0xffffffffu, y[h], o);
+            if (part == 0 && valid) {
 #pragma unroll
                 for (int h = 0; h < GMAX; ++h) {
                     if (h < G) {
-#pragma unroll
-                        for (int e = 0; e < E; e += 4) {
-                            const float4 qv = *reinterpret_cast<const float4 *>(&qs[h][c * E + e]);
-                            acc[h] = fmaf(kf[e], qv.x, acc[h]);
-                            acc[h] = fmaf(kf[e + 1], qv.y, acc[h]);
-                            acc[h] = fmaf(kf[e + 2], qv.z, acc[h]);
-                            acc[h] = fmaf(kf[e + 3], qv.w, acc[h]);
-                        }
+                        a.logits[(int64_t)(it.g * G + h) * a.total_tokens + tb.pack[it.s] + i] = y[h];
+                        if (y[h] > m[h]) { z[h] = z[h] * exp2f(m[h] - y[h]) + 1.f; m[h] = y[h]; }
+                        else z[h] += exp2f(y[h] - m[h]);
                     }
                 }
             }
         }
-        // block maximum per head, then the block's sum of 2^(y - max)
+        // block (max, sum) per head: lanes -> warp -> block, in a fixed order
 #pragma unroll
         for (int h = 0; h < GMAX; ++h) {
             if (h < G) {
-                float m = valid ? acc[h] : -INFINITY;
-                for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                if (lane == 0) red[warp][h] = m;
+                float mm = m[h];
+                for (int o = 16; o; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+                float zz = (z[h] > 0.f) ? z[h] * exp2f(m[h] - mm) : 0.f;
+                for (int o = 16; o; o >>= 1) zz += __shfl_xor_sync(0xffffffffu, zz, o);
+                if (lane == 0) red[warp][h] = make_float2(mm, zz);
             }
         }
         __syncthreads();
         if (threadIdx.x < G) {
-            float m = red[0][threadIdx.x];
-            for (int wv = 1; wv < kThreadsW1 / 32; ++wv) m = fmaxf(m, red[wv][threadIdx.x]);
-            bmax[threadIdx.x] = m;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int h = 0; h < GMAX; ++h) {
-            if (h < G) {
-                float z = valid ? exp2f(acc[h] - bmax[h]) : 0.f;
-                for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-                if (lane == 0) red[warp][h] = z;
-                if (valid)
-                    a.logits[(int64_t)(it.g * G + h) * a.total_tokens + tb.pack[it.s] + i] = acc[h];
+            float mm = -INFINITY, zz = 0.f;
+            for (int wv = 0; wv < kWarpsW1; ++wv) mm = fmaxf(mm, red[wv][threadIdx.x].x);
+            for (int wv = 0; wv < kWarpsW1; ++wv) {
+                const float2 pr = red[wv][threadIdx.x];
+                if (pr.y > 0.f) zz += pr.y * exp2f(pr.x - mm);
             }
-        }
-        __syncthreads();
-        if (threadIdx.x < G) {
-            float z = 0.f;
-            for (int wv = 0; wv < kThreadsW1 / 32; ++wv) z += red[wv][threadIdx.x];
             a.stats[((int64_t)(tb.chunks[it.s] * Hkv) + (int64_t)it.g * (tb.chunks[it.s + 1] - tb.chunks[it.s]) +
-                     it.chunk) * G + threadIdx.x] = make_float2(bmax[threadIdx.x], z);
+                     it.chunk) * G + threadIdx.x] = make_float2(mm, zz);
         }
+        __syncthreads();
     }
 }
 

@@ -190,6 +190,32 @@ refree_status refree_select_budget_static(const refree_params *p, const float *s
                                           int32_t *kept_idx, int64_t capacity_rows,
                                           int32_t *device_status, void *stream);
 
+/* Decode-step attention over the compacted ragged cache, the consumer of the
+ * pass (Algorithm 1 hands K_c, V_c to generation; Section 3.3 batches sequences
+ * whose budgets differ).  For every sequence s and query head h, with
+ * u = s*num_kv_heads + h / (num_q_heads / num_kv_heads):
+ *     out[s, h, :] = softmax(q_new[s, h, :] . K_c[rows of u]^T / sqrt(head_dim)) V_c[rows of u]
+ * over rows [offsets[u], offsets[u+1]) of k_c / v_c.
+ *   q_new    [num_seqs, num_q_heads, head_dim], params->dtype           (device, in)
+ *   k_c, v_c [rows, head_dim] contiguous, params->dtype, 16-byte aligned (device, in):
+ *            the k_out / v_out of refree_compact or refree_compress_layer
+ *   offsets  [num_seqs*num_kv_heads + 1] int64                          (device, in)
+ *   max_rows_per_unit  host-side upper bound of offsets[u+1] - offsets[u] (the longest
+ *            sequence length always is one); it sizes the launch.  A longer segment sets
+ *            REFREE_DEV_CAPACITY in *device_status and only its first rows are used.
+ *   out      [num_seqs, num_q_heads, head_dim] fp32                     (device, out);
+ *            an empty segment gives a zero row
+ *   workspace  refree_decode_workspace_size(params, max_rows_per_unit) bytes, 256-byte
+ *            aligned (device, scratch).
+ * Only num_seqs, num_q_heads, num_kv_heads, head_dim and dtype of params are read.
+ * Products are exact (bf16) or fp32, sums and the softmax are fp32. */
+refree_status refree_decode_workspace_size(const refree_params *params, int64_t max_rows_per_unit, size_t *bytes);
+refree_status refree_decode_attention(const refree_params *params, const void *q_new,
+                                      const void *k_c, const void *v_c, const int64_t *offsets,
+                                      int64_t max_rows_per_unit, float *out,
+                                      void *workspace, size_t workspace_bytes,
+                                      int32_t *device_status, void *stream);
+
 /* Diagnostic with no counterpart in the paper: the number of CUDA kernels this
  * library has enqueued in this process so far (all entry points, all streams). */
 int64_t refree_kernel_launch_count(void);

@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(HERE, "librefreekv.so")
 REFREE_OK = 0
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CAPACITY", "CUDA", "TIMEOUT", "NONFINITE",
                 "STATIC_LIMIT"]
+(ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE,
+ ERR_STATIC_LIMIT) = range(1, 9)
 STATIC_SCRATCH_BYTES = 256 * 1024
 DEV_CAPACITY, DEV_TIMEOUT, DEV_NONFINITE = 1, 2, 4
 RANK_POSITION, RANK_SCORE = 0, 1
@@ -87,6 +89,8 @@ SIGNATURES = {
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_decode_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
+    "refree_decode_attention": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
     "refree_host_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
     "refree_compress_layer_host": (ctypes.c_int, [_PP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP, _I64,
                                                   _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
@@ -203,6 +207,26 @@ def refree_compress_layer(p: Params, q_win, k, v, seq_start, seq_len, total_toke
                                      _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_compress_layer")
+    return rc
+
+
+def refree_decode_workspace_size(p: Params, max_rows_per_unit: int) -> int:
+    out = _SZ(0)
+    c = p.c_struct()
+    _check(lib().refree_decode_workspace_size(ctypes.byref(c), max_rows_per_unit, ctypes.byref(out)),
+           "refree_decode_workspace_size")
+    return int(out.value)
+
+
+def refree_decode_attention(p: Params, q_new, k_c, v_c, offsets, max_rows_per_unit, out, workspace,
+                            device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_decode_attention(ctypes.byref(c), _dp(q_new), _dp(k_c), _dp(v_c), _dp(offsets),
+                                       max_rows_per_unit, _dp(out), _dp(workspace),
+                                       workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                       _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_decode_attention")
     return rc
 
 

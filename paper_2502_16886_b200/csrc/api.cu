@@ -193,6 +193,45 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
                                     v_out, capacity_rows, device_status, (cudaStream_t)stream));
 }
 
+static refree_status check_decode(const refree_params *p, int64_t max_rows)
+{
+    if (!p) return REFREE_ERR_INVALID_ARG;
+    if (p->num_seqs < 1 || p->num_q_heads < 1 || p->num_kv_heads < 1) return REFREE_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads != 0) return REFREE_ERR_INVALID_ARG;
+    if (p->dtype != REFREE_DTYPE_F32 && p->dtype != REFREE_DTYPE_BF16) return REFREE_ERR_INVALID_ARG;
+    if (max_rows < 0 || max_rows > 0x7fffffffLL - 4096) return REFREE_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return REFREE_ERR_UNSUPPORTED;
+    if ((int64_t)p->num_seqs * p->num_kv_heads > 65535) return REFREE_ERR_UNSUPPORTED;
+    if (p->num_q_heads / p->num_kv_heads > 16) return REFREE_ERR_UNSUPPORTED;
+    return REFREE_OK;
+}
+
+refree_status refree_decode_workspace_size(const refree_params *p, int64_t max_rows_per_unit, size_t *bytes)
+{
+    const refree_status st = check_decode(p, max_rows_per_unit);
+    if (st != REFREE_OK) return st;
+    if (!bytes) return REFREE_ERR_INVALID_ARG;
+    *bytes = decode_workspace_bytes(*p, max_rows_per_unit);
+    return REFREE_OK;
+}
+
+refree_status refree_decode_attention(const refree_params *p, const void *q_new,
+                                      const void *k_c, const void *v_c, const int64_t *offsets,
+                                      int64_t max_rows_per_unit, float *out,
+                                      void *workspace, size_t workspace_bytes,
+                                      int32_t *device_status, void *stream)
+{
+    const refree_status st = check_decode(p, max_rows_per_unit);
+    if (st != REFREE_OK) return st;
+    if (!q_new || !k_c || !v_c || !offsets || !out) return REFREE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_c) & 15) || (reinterpret_cast<uintptr_t>(v_c) & 15)) return REFREE_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < decode_workspace_bytes(*p, max_rows_per_unit) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    return from_cuda(launch_decode_attention(*p, q_new, k_c, v_c, offsets, max_rows_per_unit, out, workspace,
+                                             device_status, (cudaStream_t)stream));
+}
+
 refree_status refree_compress_layer(const refree_params *p, const void *q_win,
                                     const void *k, const void *v,
                                     const int32_t *seq_start, const int32_t *seq_len,

@@ -151,4 +151,9 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            bool position_ranges, int64_t *offsets_out, void *k_out, void *v_out,
                            int64_t capacity_rows, int32_t *dev_status, cudaStream_t st);
 
+size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
+cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,
+                                    const int64_t *offsets, int64_t max_rows, float *out, void *workspace,
+                                    int32_t *dev_status, cudaStream_t st);
+
 }  // namespace refree

@@ -212,3 +212,30 @@ def make_layer(cfg: CacheConfig, layer: int, layout: str = "head_major",
     return LayerCache(cfg, layer, layout, q_all, k_all, v_all,
                       torch.tensor(starts, dtype=torch.int32),
                       torch.tensor(lens, dtype=torch.int32), heavy_all)
+
+
+def make_decode_query(cfg: CacheConfig, layer: int, q_win: torch.Tensor) -> torch.Tensor:
+    """Query of the first generated token, ``[B, Hq, d]`` in the cache dtype.
+
+    Drawn like a window row (unit-variance coordinates around the direction the
+    window queries of the head share, estimated here as their mean over the
+    window), from a generator seeded ``1_000_000*c + 1000*layer + 777``.
+    """
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(1_000_000 * cfg.index + 1000 * layer + 777)
+    mean = q_win.to(torch.float32).mean(dim=2)                      # [B, Hq, d]
+    z = torch.randn(mean.shape, generator=gen, dtype=torch.float32)
+    return (z / math.sqrt(2.0) + mean).to(cfg.torch_dtype).contiguous()
+
+
+def make_ragged_cache(seed: int, lengths, head_dim: int, dtype: torch.dtype):
+    """A dense ragged cache with the given per-unit row counts (rows ~ N(0,1)):
+    ``(k_c, v_c, offsets)`` with ``offsets`` the int64 running sum of ``lengths``."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    rows = int(sum(lengths))
+    k_c = torch.randn((max(rows, 1), head_dim), generator=gen, dtype=torch.float32).to(dtype)
+    v_c = torch.randn((max(rows, 1), head_dim), generator=gen, dtype=torch.float32).to(dtype)
+    offsets = torch.zeros(len(lengths) + 1, dtype=torch.int64)
+    offsets[1:] = torch.cumsum(torch.tensor(list(lengths), dtype=torch.int64), 0)
+    return k_c, v_c, offsets

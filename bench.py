@@ -311,6 +311,33 @@ def run_ours(args):
                      "bytes_per_layer": int(bytes3), "bytes_per_layer_with_kept_k_reread": int(bytes4),
                      "kept_ratio": round(rho, 4), "ms_per_layer": round(ms_layer, 5)}
 
+    # the consumer of the pass: one decode step of attention over every layer's compacted cache, swept like a stage
+    max_rows = max(seq_lens)
+    dws = torch.empty(binding.refree_decode_workspace_size(params, max_rows), dtype=torch.uint8, device=dev)
+    q_new = workloads.make_decode_query(cfg, 0, host0.q_win).to(dev)
+    dout = torch.empty(len(seq_lens), cfg.num_q_heads, cfg.head_dim, dtype=torch.float32, device=dev)
+
+    def decode(d):
+        binding.refree_decode_attention(params, q_new, d["k_out"], d["v_out"], d["offsets"], max_rows, dout, dws, status)
+
+    for d in layers:
+        decode(d)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        for d in layers:
+            decode(d)
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    dec_ms = e0.elapsed_time(e1) / (reps * L)
+    dec_bytes = 2 * kept_rows * row
+    dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    decode_line = {"kernel": "refree_decode_attention", "bound": "hbm", "ms_per_layer": round(dec_ms, 5),
+                   "bytes_per_layer": int(dec_bytes), "achieved": round(dec_gbs, 1), "peak": peak,
+                   "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(dec_gbs / peak, 4)}
+
     e2e = measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args)
     cpu_baseline = measure_cpu_baseline(cfg, rank_mode, total, args) if world == 1 and not args.no_cpu_baseline else None
 
@@ -326,7 +353,8 @@ def run_ours(args):
                          f"({L * 2 * cfg.num_kv_heads * total * row / 2**30:.1f} GiB), larger than L2",
                    "replicas": world},
         "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
-        "roofline": roofline, "roofline_pass": roofline_pass, "cpu_baseline": cpu_baseline,
+        "roofline": roofline, "roofline_pass": roofline_pass, "decode_attention": decode_line,
+        "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

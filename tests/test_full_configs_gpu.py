@@ -39,3 +39,29 @@ def test_layer_scope_and_frozen_layer_at_full_size():
     assert len(set(res.lengths.cpu().reshape(-1).tolist())) == 1      # one budget for the layer
     res, _, _, _ = parity.run_fused_and_check(cfg, lay, force_full=1, want_scores=False)
     assert (res.lengths == 8192).all()
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_8k", "mistral7b_32k", "qwen25_7b_ragged8", "llama3_70b_20k"])
+def test_decode_attention_over_the_compacted_layer_at_full_size(name):
+    # the consumer of the pass at benchmark size: every output element against the fp64 oracle
+    from oracle import refree_oracle as orc
+    cfg = workloads.get_config(name)
+    lay = workloads.make_layer(cfg, 0)
+    dev = "cuda:0"
+    p = binding.params_for(cfg, lay)
+    res = binding.compress_layer(p, lay.q_win.to(dev), lay.k.to(dev), lay.v.to(dev), lay.seq_start.to(dev),
+                                 lay.seq_len.to(dev), lay.total_tokens, want_scores=False, want_kept_idx=False)
+    q_new = workloads.make_decode_query(cfg, 0, lay.q_win)
+    max_rows = int(lay.seq_len.max().item())
+    ws = torch.empty(binding.refree_decode_workspace_size(p, max_rows), dtype=torch.uint8, device=dev)
+    out = torch.empty((p.num_seqs, p.num_q_heads, p.head_dim), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.refree_decode_attention(p, q_new.to(dev), res.k_out, res.v_out, res.offsets, max_rows, out, ws,
+                                    device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = int(res.offsets[-1].item())
+    op = orc.OracleParams(p.num_seqs, p.num_q_heads, p.num_kv_heads, p.head_dim, dtype=1)
+    want = orc.decode_attention(op, q_new, res.k_out[:rows].cpu(), res.v_out[:rows].cpu(), res.offsets.cpu().numpy())
+    np.testing.assert_allclose(out.cpu().numpy(), want, rtol=1e-4, atol=1e-4)
+    torch.cuda.empty_cache()

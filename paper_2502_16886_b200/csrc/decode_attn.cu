@@ -165,23 +165,30 @@ decode_mma_kernel(DecArgs a)
     for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
 
-    for (int row0 = begin + warp * 16; row0 < end; row0 += kDecWarps * 16) {
-        // K: B operand of the two S^T products (rows row0 + r and row0 + 8 + r)
-        uint4 k1[CH], k2[CH];
+    // K: B operand of the two S^T products (rows row0 + r and row0 + 8 + r);
+    // V: rows 2c, 2c + 1, 8 + 2c, 9 + 2c of the block, piece r of each 128-byte half.
+    // The registers of K are refilled for the next block as soon as the logits are formed and
+    // those of V right after the second product, so the loads fly under the other phase's math.
+    uint4 k1[CH], k2[CH], v[4][HF];
+    auto load_k = [&](int row0) {
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
             k1[j] = dec_ld16(kbase + (int64_t)(row0 + r) * D * 2 + j * 64 + c * 16, row0 + r < end);
             k2[j] = dec_ld16(kbase + (int64_t)(row0 + 8 + r) * D * 2 + j * 64 + c * 16, row0 + 8 + r < end);
         }
-        // V: rows 2c, 2c + 1, 8 + 2c, 9 + 2c of the block, piece r of each 128-byte half
-        const int vr[4] = {row0 + 2 * c, row0 + 2 * c + 1, row0 + 8 + 2 * c, row0 + 9 + 2 * c};
-        uint4 v[4][HF];
+    };
+    auto load_v = [&](int row0) {
+        const int rows[4] = {row0 + 2 * c, row0 + 2 * c + 1, row0 + 8 + 2 * c, row0 + 9 + 2 * c};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int hf = 0; hf < HF; ++hf)
-                v[i][hf] = dec_ld16(vbase + (int64_t)vr[i] * D * 2 + hf * 128 + r * 16, vr[i] < end);
-
+                v[i][hf] = dec_ld16(vbase + (int64_t)rows[i] * D * 2 + hf * 128 + r * 16, rows[i] < end);
+    };
+    if (begin + warp * 16 < end) { load_k(begin + warp * 16); load_v(begin + warp * 16); }
+    for (int row0 = begin + warp * 16; row0 < end; row0 += kDecWarps * 16) {
+        const int vr[4] = {row0 + 2 * c, row0 + 2 * c + 1, row0 + 8 + 2 * c, row0 + 9 + 2 * c};
+        const int next = row0 + kDecWarps * 16;
         float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
@@ -190,6 +197,7 @@ decode_mma_kernel(DecArgs a)
             dec_mma(s2, qa[j].x, qb[j].x, qa[j].y, qb[j].y, k2[j].x, k2[j].y);
             dec_mma(s2, qa[j].z, qb[j].z, qa[j].w, qb[j].w, k2[j].z, k2[j].w);
         }
+        if (next < end) load_k(next);
         // lane (r, c): y[hh][0..3] = logits of head r + 8 hh for rows vr[0..3]
         float y[2][4];
 #pragma unroll
@@ -242,6 +250,7 @@ decode_mma_kernel(DecArgs a)
                     dec_mma(o[t], al[0], al[1], al[2], al[3], b0, b1);
                 }
         }
+        if (next < end) load_v(next);
     }
     // the four column lanes of a head hold partial sums of l
 #pragma unroll
@@ -334,31 +343,67 @@ decode_lanes_kernel(DecArgs a)
     merge_and_store<D>(a, dec_sm, GMAX, G, u, x, nblocks);
 }
 
-// One block per (unit, head): merges the span records in span order and normalises.
+// One block per (unit, head): merges the span records and normalises.  The weights 2^(m_b - M)
+// are formed first (a thread per span), then every thread sums its column over a slice of the
+// spans with independent loads; the slices meet in shared memory in slice order.
+constexpr int kCombineThreads = 512;
+constexpr int kMaxSpans = 1024;
+
 template <int D>
-__global__ void __launch_bounds__(D)
+__global__ void __launch_bounds__(kCombineThreads)
 decode_combine_kernel(DecArgs a)
 {
+    constexpr int SL = kCombineThreads / D;         // slices of the span list
+    __shared__ float w[kMaxSpans], wl[kMaxSpans];
+    __shared__ float red[kCombineThreads / 32];
+    __shared__ float acc[SL][D];
+    __shared__ float s_M, s_L;
     const refree_params &p = a.p;
     const int Hkv = p.num_kv_heads, G = p.num_q_heads / Hkv;
     const int u = blockIdx.x / G, h = blockIdx.x % G, s = u / Hkv, g = u % Hkv;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t len64 = a.offsets[u + 1] - a.offsets[u];
     const int len = (int)max((int64_t)0, min(len64, (int64_t)a.span * a.gx));
     const int nblocks = ceil_div(len, a.span);
     if (nblocks <= 1) return;                       // written by the attention kernel itself
     const float *rec0 = a.part + ((int64_t)u * a.gx * G + h) * (D + 2);
     const int64_t stride = (int64_t)G * (D + 2);
-    float M = -INFINITY;
-    for (int b = 0; b < nblocks; ++b) M = fmaxf(M, rec0[b * stride + D]);
-    float val = 0.f, L = 0.f;
-#pragma unroll 4
-    for (int b = 0; b < nblocks; ++b) {
-        const float *rec = rec0 + b * stride;
-        const float f = dec_ex2(rec[D] - M);
-        val += rec[threadIdx.x] * f;
-        L += rec[D + 1] * f;
+    // M = max of the span maxima
+    float m = -INFINITY;
+    for (int b = tid; b < nblocks; b += kCombineThreads) m = fmaxf(m, rec0[b * stride + D]);
+    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (tid == 0) {
+        float M = -INFINITY;
+        for (int i = 0; i < kCombineThreads / 32; ++i) M = fmaxf(M, red[i]);
+        s_M = M;
     }
-    a.out[((int64_t)s * p.num_q_heads + g * G + h) * D + native_col(threadIdx.x, a.native)] = L > 0.f ? val / L : 0.f;
+    __syncthreads();
+    const float M = s_M;
+    for (int b = tid; b < nblocks; b += kCombineThreads) {
+        w[b] = dec_ex2(rec0[b * stride + D] - M);
+        wl[b] = w[b] * rec0[b * stride + D + 1];
+    }
+    __syncthreads();
+    if (tid == 0) {                                 // the denominator, in span order
+        float L = 0.f;
+        for (int b = 0; b < nblocks; ++b) L += wl[b];
+        s_L = L;
+    }
+    const int col = tid % D, sl = tid / D;
+    const int per = ceil_div(nblocks, SL), b0 = sl * per, b1 = min(nblocks, b0 + per);
+    float val = 0.f;
+#pragma unroll 8
+    for (int b = b0; b < b1; ++b) val += w[b] * rec0[b * stride + col];
+    acc[sl][col] = val;
+    __syncthreads();
+    if (tid < D) {
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < SL; ++i) tot += acc[i][tid];
+        a.out[((int64_t)s * p.num_q_heads + g * G + h) * D + native_col(tid, a.native)] = s_L > 0.f ? tot / s_L : 0.f;
+    }
 }
 
 template <typename T, int D>
@@ -397,7 +442,7 @@ cudaError_t run_mma(const DecArgs &a, dim3 grid, int G, cudaStream_t st)
 void decode_shape(const refree_params &p, int64_t max_rows, int &gx, int &span)
 {
     const int64_t U = (int64_t)p.num_seqs * p.num_kv_heads;
-    const int64_t want = std::max<int64_t>(1, (148 * 4) / U);                  // about four blocks per SM
+    const int64_t want = std::min<int64_t>(kMaxSpans, std::max<int64_t>(1, (148 * 2) / U));   // about two blocks per SM
     const int64_t by_rows = std::max<int64_t>(1, (max_rows + 127) / 128);      // at least one 16-row block per warp
     gx = (int)std::min<int64_t>(want, by_rows);
     span = (int)(((max_rows + gx - 1) / gx + 15) / 16 * 16);
@@ -441,8 +486,8 @@ cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, c
     }
     count_launches(1);
     if (e != cudaSuccess || a.gx == 1) return e;
-    if (p.head_dim == 64) decode_combine_kernel<64><<<U * G, 64, 0, st>>>(a);
-    else decode_combine_kernel<128><<<U * G, 128, 0, st>>>(a);
+    if (p.head_dim == 64) decode_combine_kernel<64><<<U * G, kCombineThreads, 0, st>>>(a);
+    else decode_combine_kernel<128><<<U * G, kCombineThreads, 0, st>>>(a);
     count_launches(1);
     return cudaGetLastError();
 }

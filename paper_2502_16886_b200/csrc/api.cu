@@ -21,9 +21,9 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     const int64_t rows = G * p.window;
     const int64_t tiles = total_tokens / kTile + p.num_seqs;
     size_t off = 0;
-    // partials: per (tile, head, row) for the generic path, per (CTA + unit, padded row) for the tensor-core path
+    // partials: per (tile, head, row) for the generic path, per (CTA + unit, column half, padded row) for the tensor-core path
     const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
-    const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, (256 + U) * rows_pad);
+    const int64_t part_items = std::max<int64_t>(tiles * p.num_kv_heads * rows, 2 * (256 + U) * rows_pad);
     size_t part_bytes = (size_t)part_items * sizeof(float2);
     if (score_w1_supported(p)) part_bytes = std::max(part_bytes, score_w1_scratch_bytes(p, total_tokens));
     w.part_off = off;   w.part_bytes = align256(part_bytes);                                               off += w.part_bytes;

@@ -16,9 +16,12 @@
 // Both passes use the same shared-memory images of Q and K (K-major, so either
 // can be the A or the B operand); only the roles swap, which puts each pass's
 // reduction inside a thread.  Persistent CTAs (one per SM) take contiguous ranges
-// of (unit, tile) items; warp 8 issues TMA, warp 9 issues MMA, warps 0-7 are the
-// epilogue (two warpgroups, each on one half of a 256-column accumulator, two
-// accumulators in flight).  Every wait is bounded: on a timeout the CTA records
+// of (unit, tile) items; warp 16 issues TMA, warp 17 issues MMA, warps 0-15 are the
+// epilogue: four warpgroups = (accumulator pair) x (64-column half of a 128-column
+// accumulator), two accumulators per pair in flight.  The exponentials bind, and with
+// four warps per scheduler instead of two their latencies overlap.  In pass 1 the two
+// halves of a row keep separate (c, Z) records; in pass 2 warpgroup 0 adds the other
+// warpgroups' column sums from shared memory.  Every wait is bounded: on a timeout the CTA records
 // REFREE_DEV_TIMEOUT, stops issuing work, and falls through to the common exit
 // where tensor memory is released.
 #include <cuda.h>
@@ -32,7 +35,8 @@
 namespace refree {
 namespace {
 
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;                 // four warpgroups: (accumulator pair) x (column half)
+constexpr int kHalfCols = 64;                 // tensor-memory columns of an accumulator per warpgroup
 constexpr int kThreadsTc = (kEpiWarps + 2) * 32;
 constexpr int kD = 128;
 constexpr int kHalfBytes = kTile * 128;          // one 64-column half of a 128-row tile: 16 KB
@@ -187,10 +191,10 @@ struct TcShape {
 struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
     uint64_t acc_full[4], acc_empty[4];       // accumulator (warpgroup * 2 + slot): 128 tensor-memory columns each
-    uint64_t half_ready[3];                   // pass 2: warpgroup 1 has staged its half of a tile
+    uint64_t half_ready[4];                   // pass 2: the other warpgroups have staged their shares of a tile
     uint32_t tmem_base;
     int abort_flag;
-    alignas(16) float stage[3][kTile];        // pass 2: warpgroup 1's partial column sums, three tiles deep
+    alignas(16) float stage[4][3][kTile];     // pass 2: partial column sums of warpgroups 1..3, four tiles deep
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
     SeqTables seq;
     int32_t start[kMaxSeqs];                  // copy of seq_start
@@ -253,7 +257,7 @@ struct TcArgs {
     refree_params p;
     TcShape sh;
     const int32_t *seq_start, *seq_len;
-    float2 *part;        // [ctas + units][Rpad]
+    float2 *part;        // [2 (ctas + units)][Rpad]: one record per (CTA, unit, column half)
     GroupPartial *groups; // nullable: per 32 positions, exact sum of squared scores for the stopping rule
     uint32_t *flags;     // fused launch: flags[c] == epoch once CTA c has written its pass-1 partials
     uint32_t epoch;
@@ -401,12 +405,11 @@ __device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, in
     const float nc = -cref;
     uint32_t ra[32], rb[32];
     tmem_ld32_issue(taddr, ra);
+    tmem_ld32_issue(taddr + 32, rb);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+    for (int c = 0; c < 2; ++c) {
+        uint32_t (&cur)[32] = c ? rb : ra;
         tmem_ld_wait(cur);
-        if (c + 1 < 4) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
             float e0 = ex2(fmaf(__uint_as_float(cur[i]), scale, nc));
@@ -426,12 +429,11 @@ __device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
     float m = -INFINITY;
     uint32_t ra[32], rb[32];
     tmem_ld32_issue(taddr, ra);
+    tmem_ld32_issue(taddr + 32, rb);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+    for (int c = 0; c < 2; ++c) {
+        uint32_t (&cur)[32] = c ? rb : ra;
         tmem_ld_wait(cur);
-        if (c + 1 < 4) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
 #pragma unroll
         for (int i = 0; i < 32; ++i)
             if (c * 32 + i < limit) m = fmaxf(m, __uint_as_float(cur[i]) * scale);
@@ -444,12 +446,12 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int wg = warp >> 2, lane_base = (warp & 3) * 32;
+    const int wg = (warp >> 2) & 1, half = warp >> 3, lane_base = (warp & 3) * 32;
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
     int cur_u = -1;
     uint32_t &cnt = es.cnt;                      // blocks this warpgroup has consumed
-    // running reference and sum of this thread's rows: row blocks wg and wg + 2
+    // running reference and sum of this thread's rows (row blocks wg and wg + 2) over its half of the columns
     float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
     int rmod[2];
     bool rvalid[2];
@@ -466,7 +468,7 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             const int rb = wg + 2 * j;
             const int row = rb * kTile + lane_base + lane;
             if (rb < sh.rblocks && row < sh.R)
-                a.part[(int64_t)(blockIdx.x + u) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
+                a.part[((int64_t)(blockIdx.x + u) * 2 + half) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
             cref[j] = -INFINITY;
             zsum[j] = 0.f;
         }
@@ -495,8 +497,9 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             } else if (!rvalid[j]) {
                 limit = 0;
             }
-            const bool uniform = __all_sync(0xffffffffu, limit == kTile);
-            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
+            limit = max(0, min(kHalfCols, limit - half * kHalfCols));   // inside this warpgroup's columns
+            const bool uniform = __all_sync(0xffffffffu, limit == kHalfCols);
+            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + (uint32_t)(half * kHalfCols) + ((uint32_t)lane_base << 16);
             bool need_max = (cref[j] == -INFINITY) && limit > 0;
             float zt = 0.f;
             for (int attempt = 0; attempt < 2; ++attempt) {
@@ -523,7 +526,7 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
 
 // Pass 2: thread = position.  Sum over the rows that see it of 2^(y - L[row]).
 // One accumulator's share of a warpgroup: ncol_wg columns (a multiple of 16, at most
-// 128) taken in chunks of 32 (the last may be 16), next chunk in flight.
+// 64) in two chunks of up to 32, both loads in flight.
 template <bool MASKED>
 __device__ inline float col_sum_job(uint32_t taddr, float scale, const float *lse, int rbase, int ncol_wg,
                                     int w, int pos_gap)
@@ -532,16 +535,12 @@ __device__ inline float col_sum_job(uint32_t taddr, float scale, const float *ls
     uint32_t ra[32] = {}, rb[32] = {};
     float s0 = 0.f, s1 = 0.f;
     if (ncol_wg >= 32) tmem_ld32_issue(taddr, ra); else tmem_ld16_issue(taddr, ra);
+    if (ncol_wg >= 64) tmem_ld32_issue(taddr + 32, rb); else if (ncol_wg > 32) tmem_ld16_issue(taddr + 32, rb);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
         if (c * 32 < ncol_wg) {
-            uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-            uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+            uint32_t (&cur)[32] = c ? rb : ra;
             tmem_ld_wait(cur);
-            if (c + 1 < 4 && (c + 1) * 32 < ncol_wg) {
-                if (ncol_wg - (c + 1) * 32 >= 32) tmem_ld32_issue(taddr + (c + 1) * 32, nxt);
-                else tmem_ld16_issue(taddr + (c + 1) * 32, nxt);
-            }
             const int r0 = rbase + c * 32;
             const int width = min(32, ncol_wg - c * 32);
             int rloc = MASKED ? r0 % w : 0;
@@ -581,8 +580,9 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int wg = warp >> 2, lane_base = (warp & 3) * 32;
-    const int tid = threadIdx.x;                                   // 0..255
+    const int grp = warp >> 2;                                     // 0 finishes the tile, 1..3 stage their shares
+    const int wg = grp & 1, half = grp >> 1, lane_base = (warp & 3) * 32;
+    const int tid = threadIdx.x;                                   // 0..511
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
     const int pos_in_tile = lane_base + lane;
@@ -590,7 +590,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     int cur_u = -1;
     uint32_t &cnt = es.cnt, &ephase = es.ephase;                   // blocks consumed, phase of the epilogue barrier
     uint32_t tcount = 0;                                           // tiles seen
-    // warpgroup 0 finishes a tile one tile late, when warpgroup 1's half has long been staged
+    // warpgroup 0 finishes a tile one tile late, when the other warpgroups' shares have long been staged
     float pend_acc = 0.f, pend_norm = 0.f;
     float *pend_dst = nullptr;
     GroupPartial *pend_grp = nullptr;
@@ -599,10 +599,9 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
     auto finish_pending = [&]() -> bool {
         if (!pending) return true;
         float tot = pend_acc;
-        if (two_halves) {
-            if (!mbar_wait(&tl.half_ready[pend_tile % 3u], (pend_tile / 3u) & 1u, &tl.abort_flag)) return false;
-            tot += tl.stage[pend_tile % 3u][pos_in_tile];
-        }
+        if (!mbar_wait(&tl.half_ready[pend_tile & 3u], (pend_tile >> 2) & 1u, &tl.abort_flag)) return false;
+        tot += tl.stage[pend_tile & 3u][1][pos_in_tile];                       // same accumulators, other columns
+        if (two_halves) tot += tl.stage[pend_tile & 3u][0][pos_in_tile] + tl.stage[pend_tile & 3u][2][pos_in_tile];
         float sc = 0.f;
         if (pend_dst) {
             sc = tot * pend_norm;
@@ -648,11 +647,12 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             }
             for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
                 float M = -INFINITY, Z = 0.f;
-                for (int c0 = c_lo; c0 <= c_hi; c0 += 8) {
+                const int s_hi = 2 * (c_hi + it.u) + 1;             // records: (CTA, column half)
+                for (int s0 = 2 * (c_lo + it.u); s0 <= s_hi; s0 += 8) {
                     float2 pr[8];                                  // eight independent loads in flight
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
-                        pr[q] = (c0 + q <= c_hi) ? __ldcg(&a.part[(int64_t)(c0 + q + it.u) * sh.Rpad + r])
+                        pr[q] = (s0 + q <= s_hi) ? __ldcg(&a.part[(int64_t)(s0 + q) * sh.Rpad + r])
                                                  : make_float2(-INFINITY, 0.f);
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -667,9 +667,6 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!(ok = epi_sync(tl, ephase))) break;
             cur_u = it.u;
         }
-        // the previous tile is completed before any accumulator of this tile is handed back, which
-        // keeps warpgroup 1 at most two tiles ahead of the staging slot being read here
-        if (wg == 0 && !(ok = finish_pending())) break;
         const int i = it.tile_start + pos_in_tile;
         const int pos_gap = i - (it.n - w);
         // tile wholly before the window and wholly inside the sequence: every row sees every position
@@ -684,15 +681,22 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
             if (!ok) continue;
             ++cnt;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + ((uint32_t)lane_base << 16);
-            accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap)
-                         : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol, sh.ncol, w, pos_gap);
+            const int c_off = half * kHalfCols, ncol_h = max(0, min(kHalfCols, sh.ncol - c_off));
+            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + (uint32_t)c_off + ((uint32_t)lane_base << 16);
+            if (ncol_h > 0)
+                accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol + c_off, ncol_h, w, pos_gap)
+                             : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol + c_off, ncol_h, w, pos_gap);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
         }
         if (!ok) break;
-        if (wg == 0) {
+        // Warpgroup 0 completes the previous tile only now, after it has handed this tile's accumulators
+        // back, so the MMA of the tile after next overlaps the completion.  The others can then be at most
+        // three tiles past the staging slot read here (the accumulators of tile t + 3 need this warpgroup's
+        // release of tile t + 1, which comes after this point): four slots.
+        if (grp == 0 && !(ok = finish_pending())) break;
+        if (grp == 0) {
             const int cnt_i = max(1, min(min(w, it.n), it.n - i));
             pend_acc = accv;
             pend_norm = 1.f / ((float)cnt_i * (float)G);
@@ -702,14 +706,15 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t 
                                 : nullptr;
             pend_tile = tcount;
             pending = true;
-        } else if (two_halves) {
-            tl.stage[tcount % 3u][pos_in_tile] = accv;
+        } else if (wg == 0 || two_halves) {
+            // the second accumulator pair has blocks (and is paced by the MMA warp) only with several column blocks
+            tl.stage[tcount & 3u][grp - 1][pos_in_tile] = accv;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.half_ready[tcount % 3u]);
+            if (lane == 0) mbar_arrive(&tl.half_ready[tcount & 3u]);
         }
         ++tcount;
     }
-    if (wg == 0 && ok) finish_pending();
+    if (grp == 0 && ok) finish_pending();
 }
 
 // ---------------------------------------------------------------- kernels ----
@@ -734,7 +739,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         mbar_init(&tl.q_full, 1);
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
-        for (int b = 0; b < 3; ++b) mbar_init(&tl.half_ready[b], kEpiWarps / 2);
+        // stagers: the other column half of the first accumulator pair, plus both halves of the second pair
+        for (int b = 0; b < 4; ++b) mbar_init(&tl.half_ready[b], a.sh.cblocks > 1 ? 12 : 4);
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();

@@ -175,6 +175,18 @@ def algorithmic_bytes(cfg, seq_lens, lengths):
     return a, b4
 
 
+# dram__bytes_read + dram__bytes_write of one launch of the scoring kernel (ncu capture of the 8K workload,
+# summary under profiles/); traffic grows in proportion to the tokens, so the 32K figure is 4x the captured one.
+# Only for the kernel version the capture was taken on: window 64, tensor-core path.
+NCU_SCORE_TRAFFIC = {"llama3_8b_8k": 17_484_288, "mistral7b_32k": 4 * 17_484_288}
+
+
+def ncu_traffic(cfg, stage):
+    if stage != "score" or cfg.window != 64:
+        return None
+    return NCU_SCORE_TRAFFIC.get(cfg.name)
+
+
 def run_ours(args):
     from paper_2502_16886_b200 import binding, build, workloads
     rank, local_rank, world = dist_setup("nccl")
@@ -302,7 +314,7 @@ def run_ours(args):
     dom_gbs = stage_bytes[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
     roofline = {"kernel": f"refree_{dominant} stage", "bound": "hbm", "achieved": round(dom_gbs, 1),
                 "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(dom_gbs / peak, 4),
-                "traffic": None, "bytes_per_launch": int(stage_bytes[dominant]),
+                "traffic": ncu_traffic(cfg, dominant), "bytes_per_launch": int(stage_bytes[dominant]),
                 "ms_per_launch": round(stage_ms[dominant], 5),
                 "stages_ms": {k: round(v, 5) for k, v in stage_ms.items()},
                 "stages_gbs": {k: round(stage_bytes[k] / (stage_ms[k] * 1e-3) / 1e9, 1) for k in stage_ms}}

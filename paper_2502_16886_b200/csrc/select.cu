@@ -572,28 +572,52 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     v.heads = layer ? Hkv : 1;
     v.n = n; v.lead = lead; v.w_eff = w_eff;
     v.sbias = cut.sbias;
-    int base = 0, tie_base = 0;
-    for (int i0 = 0; i0 < n; i0 += kThreads) {
-        const int i = i0 + threadIdx.x;
-        int tie = 0, keep = 0;
-        if (i < n) {
-            if (i < lead) {
-                keep = i < cut.prot_kept;
-            } else if (i >= n - w_eff) {
-                keep = lead + (i - (n - w_eff)) < cut.prot_kept;
-            } else {
-                const u64 key = key_at(v, i);
-                keep = key > cut.tau;
-                tie = key == cut.tau;
-            }
+    // Every thread owns a run of consecutive positions, so two block scans order the whole unit:
+    // ties first (which of the positions at the crossing key are kept: the lowest indices), then
+    // the kept positions.  Runs of up to 64 positions keep their classification in two bit masks;
+    // longer ones are classified again on each walk.
+    const int run = ceil_div(n, kThreads);
+    const int lo = min(n, (int)threadIdx.x * run), hi = min(n, lo + run);
+    auto classify = [&](int i, int &sure, int &tie) {
+        sure = 0; tie = 0;
+        if (i < lead) {
+            sure = i < cut.prot_kept;
+        } else if (i >= n - w_eff) {
+            sure = lead + (i - (n - w_eff)) < cut.prot_kept;
+        } else {
+            const u64 key = key_at(v, i);
+            sure = key > cut.tau;
+            tie = key == cut.tau;
         }
-        int tie_tot, keep_tot;
-        const int tie_rank = tie_base + block_excl_scan<int>(tie, ibuf, tie_tot);
-        if (tie && tie_rank < cut.ties) keep = 1;
-        const int slot = base + block_excl_scan<int>(keep, ibuf, keep_tot);
-        if (keep && slot < b) dst[slot] = i;
-        base += keep_tot;
-        tie_base += tie_tot;
+    };
+    const bool masks = run <= 64;
+    u64 sure_m = 0ull, tie_m = 0ull;
+    int ties = 0;
+    for (int i = lo; i < hi; ++i) {
+        int sure, tie;
+        classify(i, sure, tie);
+        if (masks) { sure_m |= (u64)sure << (i - lo); tie_m |= (u64)tie << (i - lo); }
+        ties += tie;
+    }
+    int tie_tot, keep_tot;
+    int tie_rank = block_excl_scan<int>(ties, ibuf, tie_tot);
+    const int tie_rank0 = tie_rank;
+    int keeps = 0;
+    for (int i = lo; i < hi; ++i) {
+        int sure, tie;
+        if (masks) { sure = (int)((sure_m >> (i - lo)) & 1ull); tie = (int)((tie_m >> (i - lo)) & 1ull); }
+        else classify(i, sure, tie);
+        if (tie && tie_rank++ < cut.ties) sure = 1;
+        if (masks && sure) sure_m |= 1ull << (i - lo);
+        keeps += sure;
+    }
+    int slot = block_excl_scan<int>(keeps, ibuf, keep_tot);
+    tie_rank = tie_rank0;
+    for (int i = lo; i < hi; ++i) {
+        int sure, tie = 0;
+        if (masks) sure = (int)((sure_m >> (i - lo)) & 1ull);
+        else { classify(i, sure, tie); if (tie && tie_rank++ < cut.ties) sure = 1; }
+        if (sure) { if (slot < b) dst[slot] = i; ++slot; }
     }
 }
 

@@ -24,12 +24,17 @@
 // histograms of counts and of sums of squares.
 #include <algorithm>
 
+#include <cooperative_groups.h>
+
 #include "refree_internal.cuh"
 
 namespace refree {
 namespace {
 
+namespace cg = cooperative_groups;
+
 constexpr int kThreads = 1024;
+constexpr int kMaxCluster = 8;     // blocks of a thread-block cluster that share one unit in score ranking
 constexpr int kWarps = kThreads / 32;
 typedef unsigned long long u64;
 
@@ -102,6 +107,23 @@ template <typename Tv, typename Op> __device__ inline Tv block_reduce(Tv x, Tv *
     for (int wv = 1; wv < kWarps; ++wv) r = op(r, buf[wv]);
     return r;
 }
+// Values combined over the blocks of a cluster through distributed shared memory: every block
+// publishes its share, all read all shares in rank order (so all get the same result), and a
+// second barrier keeps the slot from being rewritten early.  With one block these are no-ops.
+template <typename Tv, typename Op>
+__device__ inline Tv cluster_combine(cg::cluster_group &cl, Tv *slot, Tv mine, Op op)
+{
+    const unsigned int nb = cl.num_blocks();
+    if (nb == 1) return mine;
+    if (threadIdx.x == 0) *slot = mine;
+    cl.sync();
+    Tv r = *cl.map_shared_rank(slot, 0);
+    for (unsigned int b = 1; b < nb; ++b) r = op(r, *cl.map_shared_rank(slot, b));
+    cl.sync();
+    return r;
+}
+struct AddOpU64 { __device__ unsigned long long operator()(unsigned long long a, unsigned long long b) const { return a + b; } };
+
 struct MinOp { __device__ int operator()(int a, int b) const { return min(a, b); } };
 struct MaxOpU { __device__ uint32_t operator()(uint32_t a, uint32_t b) const { return max(a, b); } };
 struct AddOpF { __device__ float operator()(float a, float b) const { return a + b; } };
@@ -192,6 +214,10 @@ struct SelectSmem {
     u64 wsum[kWarps][257];
     int pack;
     u64 c_min;
+    // cluster exchange: what this block contributes, read by every block of the cluster
+    u64 x_u64;
+    float x_f32;
+    uint32_t x_u32;
     // radix state
     u64 prefix, above_sum;
     unsigned int above_cnt;
@@ -199,12 +225,14 @@ struct SelectSmem {
 };
 
 // Fixed point of a unit: returns false when every score is zero (C_n = 0).
-__device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *dev_status)
+__device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *dev_status, cg::cluster_group &cl)
 {
+    // the blocks of a cluster take the positions in interleaved runs of 8 * kThreads
+    const int first = (int)cl.block_rank() * kThreads * 8 + threadIdx.x, step = (int)cl.num_blocks() * kThreads * 8;
     uint32_t mx = 0;
     bool bad = false;
     for (int h = 0; h < v.heads; ++h)
-        for (int i = threadIdx.x; i < v.n; i += kThreads * 8) {
+        for (int i = first; i < v.n; i += step) {
             uint32_t b[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -214,13 +242,14 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
         }
     if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
     mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
+    mx = cluster_combine<uint32_t>(cl, &sm.x_u32, mx, MaxOpU());
     if (mx == 0u) return false;
     const int emax = max(1, (int)(mx >> 23));
     // approximate sum of squares of the scores scaled into [0, 2): only its binary order of magnitude is used
     const float f = ldexpf(1.0f, 127 - emax);
     float acc = 0.f;
     for (int h = 0; h < v.heads; ++h)
-        for (int i = threadIdx.x; i < v.n; i += kThreads * 8) {
+        for (int i = first; i < v.n; i += step) {
             uint32_t b[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -232,6 +261,7 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
             }
         }
     acc = block_reduce<float>(acc, sm.fbuf, AddOpF());
+    acc = cluster_combine<float>(cl, &sm.x_f32, acc, AddOpF());
     // C_n = acc * 2^(2 (emax - 127)); put C_n * 2^S in [2^60, 2^61)
     const int S = 60 - ilogbf(fmaxf(acc, 0.25f)) - 2 * (emax - 127);
     v.sbias = S - 300;
@@ -254,10 +284,13 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
 {
     extern __shared__ __align__(16) unsigned char select_smem_raw[];
     SelectSmem &sm = *reinterpret_cast<SelectSmem *>(select_smem_raw);
+    cg::cluster_group cl = cg::this_cluster();
+    const int nblk = (int)cl.num_blocks(), rank = (int)cl.block_rank();    // > 1 only with score ranking
+    const int unit = blockIdx.x / nblk;
     const int Hkv = p.num_kv_heads;
     const bool layer = p.scope == REFREE_SCOPE_LAYER;
-    const int s = layer ? blockIdx.x : blockIdx.x / Hkv;
-    const int g = layer ? 0 : blockIdx.x % Hkv;
+    const int s = layer ? unit : unit / Hkv;
+    const int g = layer ? 0 : unit % Hkv;
     if (threadIdx.x == 0) {
         int a = 0;
         for (int t = 0; t < s; ++t) a += max(seq_len[t], 0);
@@ -278,7 +311,7 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     Cut cut;
     cut.b = n; cut.ties = 0; cut.tau = 0; cut.prot_kept = 0; cut.sbias = 0;
 
-    if (n > 0 && !p.force_full && choose_fixed_point(v, sm, dev_status)) {
+    if (n > 0 && !p.force_full && choose_fixed_point(v, sm, dev_status, cl)) {
         cut.sbias = v.sbias;
         if (p.rank_mode == REFREE_RANK_POSITION) {
             // one pass in rank order gives C_n and the warp prefixes the search needs
@@ -292,9 +325,18 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
             if (v.lead + v.w_eff >= n) { v.lead = n; v.w_eff = 0; }
             const int prot = v.lead + v.w_eff;
             u64 Cn;
-            {   // C_n over every position (the order does not matter for an integer sum)
-                UnitView all = v; all.lead = n; all.w_eff = 0;
-                Cn = range_totals(all, 0, n, ProtRank(), sm.wpre);
+            {   // C_n over every position (the order does not matter for an integer sum): this block's share
+                u64 local = 0;
+                for (int i = rank * kThreads * 8 + threadIdx.x; i < n; i += nblk * kThreads * 8) {
+                    u64 x[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) x[q] = (i + q * kThreads < n) ? sq_at(v, i + q * kThreads) : 0ull;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) local += x[q];
+                }
+                u64 tot;
+                block_excl_scan<u64>(local, sm.ubuf, tot);
+                Cn = cluster_combine<u64>(cl, &sm.x_u64, tot, AddOpU64());
             }
             if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
             __syncthreads();
@@ -323,7 +365,7 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
                     }
                     __syncthreads();
                     const u64 prefix = sm.prefix;
-                    for (int i0 = v.lead + threadIdx.x; i0 < n - v.w_eff; i0 += kThreads * 4) {
+                    for (int i0 = v.lead + rank * kThreads * 4 + threadIdx.x; i0 < n - v.w_eff; i0 += nblk * kThreads * 4) {
                         u64 key[4], val[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
@@ -350,6 +392,21 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
                         sm.hsum[threadIdx.x] = sumv;
                     }
                     __syncthreads();
+                    if (nblk > 1) {
+                        // the digit histograms of the cluster's blocks add up (integers: any order); every
+                        // block then takes the same decision from the same totals
+                        cl.sync();
+                        unsigned int c = 0u;
+                        u64 sumv = 0ull;
+                        if (threadIdx.x < 256)
+                            for (int b = 0; b < nblk; ++b) {
+                                c += cl.map_shared_rank(sm.hcnt, b)[threadIdx.x];
+                                sumv += cl.map_shared_rank(sm.hsum, b)[threadIdx.x];
+                            }
+                        cl.sync();
+                        if (threadIdx.x < 256) { sm.hcnt[threadIdx.x] = c; sm.hsum[threadIdx.x] = sumv; }
+                        __syncthreads();
+                    }
                     // inclusive sums from the top digit down; thread t owns digit 255 - t
                     u64 mysum = 0ull, tot_s;
                     unsigned int mycnt = 0u, tot_c;
@@ -389,7 +446,8 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
             }
         }
     }
-    if (threadIdx.x == 0) {
+    if (nblk > 1) cl.sync();               // no block exits while another may still read its shared memory
+    if (threadIdx.x == 0 && rank == 0) {
         const int g_hi = layer ? Hkv : g + 1;
         for (int gg = g; gg < g_hi; ++gg) {
             lengths[s * Hkv + gg] = cut.b;
@@ -641,9 +699,39 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     }
     if (groups && p.rank_mode == REFREE_RANK_POSITION && p.scope == REFREE_SCOPE_HEAD && !p.force_full)
         select_groups_kernel<<<U, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, groups, lengths, cuts);
-    else
-        select_budget_kernel<<<sel_units, kThreads, sizeof(SelectSmem), st>>>(p, scores, seq_len, total_tokens, lengths,
-                                                                                cuts, dev_status);
+    else {
+        // score ranking walks every score several times: a cluster of blocks shares a unit (distributed
+        // shared memory for the few totals they exchange); position ranking keeps one block per unit
+        int nblk = 1;
+        if (p.rank_mode == REFREE_RANK_SCORE && !p.force_full) {
+            const int64_t avg = total_tokens / std::max(1, p.num_seqs);
+            while (nblk < kMaxCluster && avg >= (int64_t)nblk * 4096) nblk *= 2;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(sel_units * nblk);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = sizeof(SelectSmem);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = nblk;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (nblk > 1) {
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, select_budget_kernel, &cfg) != cudaSuccess || clusters < 1) {
+                (void)cudaGetLastError();
+                nblk = 1;
+                cfg.gridDim = dim3(sel_units);
+                attr[0].val.clusterDim.x = 1;
+            }
+        }
+        const cudaError_t le = cudaLaunchKernelEx(&cfg, select_budget_kernel, p, scores, seq_len, total_tokens, lengths,
+                                                  cuts, dev_status);
+        if (le != cudaSuccess) return le;
+    }
     if (!emit) {               // the caller forms the offsets itself and needs no index list
         count_launches(1);
         return cudaGetLastError();

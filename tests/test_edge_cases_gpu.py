@@ -1,0 +1,94 @@
+"""Edge cases of the pass on the GPU, each through every scoring path (tensor-core,
+single query row, generic) and both rankings: empty sequences inside a batch, the
+largest row counts each path takes, and score ranking when a cluster of blocks
+shares a unit whose sequences are far shorter than the batch mean."""
+import dataclasses
+
+import pytest
+import torch
+
+from paper_2502_16886_b200 import binding, build, workloads
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.lib()
+
+
+def cfg_like(**kw):
+    return dataclasses.replace(workloads.CONFIGS[0], **kw)
+
+
+@pytest.mark.parametrize("rank_mode", [binding.RANK_POSITION, binding.RANK_SCORE])
+@pytest.mark.parametrize("path", ["generic_fp32", "tensor_core", "single_row"])
+def test_empty_sequences_inside_a_batch(path, rank_mode):
+    if path == "generic_fp32":
+        cfg = cfg_like(num_q_heads=4, num_kv_heads=2, window=8)
+    elif path == "tensor_core":
+        cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2, window=16)
+    else:
+        cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2, window=1)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[0, 300, 0, 0, 5, 129, 0])
+    res, ref, _, _ = parity.run_fused_and_check(cfg, lay, rank_mode=rank_mode)
+    lengths = res.lengths.cpu()
+    assert (lengths[[0, 2, 3, 6]] == 0).all()           # an empty sequence keeps nothing
+    assert (lengths[[1, 4, 5]] >= 1).all()
+
+
+def test_batch_of_only_empty_sequences():
+    # the cache buffers exist (16 rows) but every sequence is empty: nothing kept, nothing written
+    dev = torch.device("cuda:0")
+    hq, hkv, d, w, rows = 4, 2, 64, 8, 16
+    p = binding.Params(num_seqs=2, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, window=w, dtype=binding.DTYPE_F32,
+                       kv_tokens=rows, k_strides=(0, d, rows * d), v_strides=(0, d, rows * d))
+    k = torch.randn(hkv, rows, d, device=dev)
+    v = torch.randn(hkv, rows, d, device=dev)
+    q = torch.randn(2, hq, w, d, device=dev)
+    zeros = torch.zeros(2, dtype=torch.int32, device=dev)
+    res = binding.compress_layer(p, q, k, v, zeros, zeros, 0, capacity_rows=4)
+    torch.cuda.synchronize()
+    assert int(res.device_status.item()) == 0
+    assert (res.lengths == 0).all() and (res.offsets == 0).all()
+
+
+@pytest.mark.parametrize("hq,hkv,w", [(8, 1, 64), (16, 2, 64), (4, 1, 128)])
+def test_largest_row_count_of_the_tensor_core_path(hq, hkv, w):
+    # G * w = 512 rows: four row blocks in pass 1, four column blocks in pass 2
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=hq, num_kv_heads=hkv, window=w)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[1000, 77])
+    parity.run_fused_and_check(cfg, lay)
+    parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE)
+
+
+def test_largest_row_count_of_the_generic_path():
+    # G * w = 1024 rows, fp32
+    cfg = cfg_like(num_q_heads=8, num_kv_heads=1, window=128)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[400, 130])
+    parity.run_fused_and_check(cfg, lay)
+
+
+def test_sixteen_query_heads_per_kv_head_single_row():
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=32, num_kv_heads=2, window=1)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[2000, 33])
+    parity.run_fused_and_check(cfg, lay)
+
+
+@pytest.mark.parametrize("scope", [binding.SCOPE_HEAD, binding.SCOPE_LAYER])
+@pytest.mark.parametrize("threshold", [0.01, 0.2])
+def test_score_ranking_with_a_cluster_per_unit_on_a_ragged_batch(scope, threshold):
+    # the mean length (about 10 K) puts two blocks on every unit, also on the sequences of 1, 40 and
+    # 300 positions, where all but one block of the cluster have no positions at all
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2, window=16, heavy_count=40)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[30000, 300, 1, 20000, 40])
+    parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE, scope=scope, threshold=threshold)
+
+
+def test_score_ranking_with_eight_blocks_per_unit():
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=4, num_kv_heads=1, window=32, heavy_count=200)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[40000])
+    parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE)
+    parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE, scope=binding.SCOPE_LAYER, threshold=0.05)

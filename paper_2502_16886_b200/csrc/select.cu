@@ -630,14 +630,16 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     v.heads = layer ? Hkv : 1;
     v.n = n; v.lead = lead; v.w_eff = w_eff;
     v.sbias = cut.sbias;
-    // Every thread owns a run of consecutive positions, so two block scans order the whole unit:
-    // ties first (which of the positions at the crossing key are kept: the lowest indices), then
-    // the kept positions.  Runs of up to 64 positions keep their classification in two bit masks;
-    // longer ones are classified again on each walk.
-    const int run = ceil_div(n, kThreads);
-    const int lo = min(n, (int)threadIdx.x * run), hi = min(n, lo + run);
-    auto classify = [&](int i, int &sure, int &tie) {
-        sure = 0; tie = 0;
+    // Every warp owns a range of consecutive positions and walks it 32 at a time (coalesced loads);
+    // votes give the order inside a step, running counts the order inside the warp, and two block
+    // scans over the warps' totals the order inside the unit: ties first (which of the positions at
+    // the crossing key are kept: the lowest indices), then the kept positions.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int span = ceil_div(ceil_div(n, kWarps), 32) * 32;
+    const int lo = min(n, warp * span), hi = min(n, lo + span);
+    auto classify = [&](int i, bool &sure, bool &tie) {
+        sure = false; tie = false;
+        if (i >= hi) return;
         if (i < lead) {
             sure = i < cut.prot_kept;
         } else if (i >= n - w_eff) {
@@ -648,34 +650,38 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
             tie = key == cut.tau;
         }
     };
-    const bool masks = run <= 64;
-    u64 sure_m = 0ull, tie_m = 0ull;
     int ties = 0;
-    for (int i = lo; i < hi; ++i) {
-        int sure, tie;
-        classify(i, sure, tie);
-        if (masks) { sure_m |= (u64)sure << (i - lo); tie_m |= (u64)tie << (i - lo); }
-        ties += tie;
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        bool sure, tie;
+        classify(i0 + lane, sure, tie);
+        ties += __popc(__ballot_sync(0xffffffffu, tie));
     }
     int tie_tot, keep_tot;
-    int tie_rank = block_excl_scan<int>(ties, ibuf, tie_tot);
+    const int tie_base = block_excl_scan<int>(lane == 0 ? ties : 0, ibuf, tie_tot);   // lane 0 carries the warp's count
+    int tie_rank = __shfl_sync(0xffffffffu, tie_base, 0);
     const int tie_rank0 = tie_rank;
     int keeps = 0;
-    for (int i = lo; i < hi; ++i) {
-        int sure, tie;
-        if (masks) { sure = (int)((sure_m >> (i - lo)) & 1ull); tie = (int)((tie_m >> (i - lo)) & 1ull); }
-        else classify(i, sure, tie);
-        if (tie && tie_rank++ < cut.ties) sure = 1;
-        if (masks && sure) sure_m |= 1ull << (i - lo);
-        keeps += sure;
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        bool sure, tie;
+        classify(i0 + lane, sure, tie);
+        const unsigned int tm = __ballot_sync(0xffffffffu, tie);
+        if (tie && tie_rank + __popc(tm & ((1u << lane) - 1u)) < cut.ties) sure = true;
+        tie_rank += __popc(tm);
+        keeps += __popc(__ballot_sync(0xffffffffu, sure));
     }
-    int slot = block_excl_scan<int>(keeps, ibuf, keep_tot);
+    const int keep_base = block_excl_scan<int>(lane == 0 ? keeps : 0, ibuf, keep_tot);
+    int slot = __shfl_sync(0xffffffffu, keep_base, 0);
     tie_rank = tie_rank0;
-    for (int i = lo; i < hi; ++i) {
-        int sure, tie = 0;
-        if (masks) sure = (int)((sure_m >> (i - lo)) & 1ull);
-        else { classify(i, sure, tie); if (tie && tie_rank++ < cut.ties) sure = 1; }
-        if (sure) { if (slot < b) dst[slot] = i; ++slot; }
+    for (int i0 = lo; i0 < hi; i0 += 32) {
+        bool sure, tie;
+        classify(i0 + lane, sure, tie);
+        const unsigned int tm = __ballot_sync(0xffffffffu, tie);
+        if (tie && tie_rank + __popc(tm & ((1u << lane) - 1u)) < cut.ties) sure = true;
+        tie_rank += __popc(tm);
+        const unsigned int km = __ballot_sync(0xffffffffu, sure);
+        const int mine = slot + __popc(km & ((1u << lane) - 1u));
+        if (sure && mine < b) dst[mine] = i0 + lane;
+        slot += __popc(km);
     }
 }
 

@@ -6,9 +6,10 @@
 //
 // The step streams K_c and V_c once (G query heads share every row): HBM-bound.
 //
-//   bf16   block = (unit, span of rows), eight warps take 16-row blocks round-robin.
-//          mma.m16n8k16 serves as the dot-product unit, fed from global memory without
-//          a shared-memory stage:
+//   bf16   block = (unit, span of rows), eight warps take 16-row blocks round-robin.  A block
+//          of 16 rows is contiguous in the compacted cache: one lane of the warp copies it with
+//          cp.async.bulk into the warp's private shared-memory ring (three blocks in flight,
+//          mbarrier-signalled).  mma.m16n8k16 serves as the dot-product unit:
 //            S^T[head, row] = Q K^T   A = the G (<= 16) queries, B = 8 rows of K; each
 //                                     lane reads 16-byte pieces of "its" row and the
 //                                     queries are cut the same way, so the order of the
@@ -34,6 +35,7 @@ namespace {
 constexpr int kDecThreads = 256;
 constexpr int kDecWarps = kDecThreads / 32;
 constexpr float kLog2eDec = 1.4426950408889634f;
+constexpr int kDecStages = 3;       // 16-row blocks of K and V in flight per warp
 
 struct DecArgs {
     refree_params p;
@@ -68,6 +70,37 @@ __device__ inline uint4 dec_ld16(const char *p, bool valid)
         asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
+}
+
+// ---- per-warp staging ring: bulk copies (TMA engine, no tensor map) signalled on an mbarrier ----
+__device__ inline uint32_t dec_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ inline void dec_bar_init(uint64_t *bar)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(dec_smem(bar)) : "memory");
+}
+__device__ inline void dec_bar_expect(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(dec_smem(bar)), "r"(bytes) : "memory");
+}
+// contiguous global -> shared copy; addresses 16-byte aligned, size a multiple of 16
+__device__ inline void dec_bulk_copy(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dec_smem(dst)), "l"(src), "r"(bytes), "r"(dec_smem(bar)) : "memory");
+}
+// bounded wait for the phase with the given parity; false when it gave up
+__device__ inline bool dec_bar_wait(uint64_t *bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(dec_smem(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+        if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
+    }
+    return false;
 }
 
 // p = hi + lo with hi, lo bf16: packs two probabilities per register for the A operand
@@ -167,28 +200,46 @@ decode_mma_kernel(DecArgs a)
 
     // K: B operand of the two S^T products (rows row0 + r and row0 + 8 + r);
     // V: rows 2c, 2c + 1, 8 + 2c, 9 + 2c of the block, piece r of each 128-byte half.
-    // The registers of K are refilled for the next block as soon as the logits are formed and
-    // those of V right after the second product, so the loads fly under the other phase's math.
-    uint4 k1[CH], k2[CH], v[4][HF];
-    auto load_k = [&](int row0) {
+    // A 16-row block of K (and of V) is contiguous in the compacted cache, so one lane brings it in
+    // with a bulk copy into the warp's own ring: kDecStages blocks per warp are in flight at the
+    // price of two instructions each (registers could hold one, and per-lane cp.async costs more
+    // to issue than the products of the block).  The ring is private to the warp: its lanes wait on
+    // the warp's barriers and lane 0 refills a slot after all lanes have read it.
+    constexpr int kBlockBytes = 16 * D * 2;          // one 16-row block of K (or V)
+    unsigned char *ring = reinterpret_cast<unsigned char *>(dec_sm) + (size_t)warp * kDecStages * 2 * kBlockBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(dec_sm) +
+                                                  (size_t)kDecWarps * kDecStages * 2 * kBlockBytes) + warp * kDecStages;
+    if (lane == 0) {
 #pragma unroll
-        for (int j = 0; j < CH; ++j) {
-            k1[j] = dec_ld16(kbase + (int64_t)(row0 + r) * D * 2 + j * 64 + c * 16, row0 + r < end);
-            k2[j] = dec_ld16(kbase + (int64_t)(row0 + 8 + r) * D * 2 + j * 64 + c * 16, row0 + 8 + r < end);
+        for (int st = 0; st < kDecStages; ++st) dec_bar_init(bars + st);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    auto issue = [&](int row0, int slot) {           // lane 0 only
+        if (row0 < end) {
+            const uint32_t bytes = (uint32_t)min(16, end - row0) * D * 2;
+            dec_bar_expect(bars + slot, 2 * bytes);
+            dec_bulk_copy(ring + (size_t)slot * 2 * kBlockBytes, kbase + (int64_t)row0 * D * 2, bytes, bars + slot);
+            dec_bulk_copy(ring + (size_t)slot * 2 * kBlockBytes + kBlockBytes, vbase + (int64_t)row0 * D * 2, bytes, bars + slot);
         }
     };
-    auto load_v = [&](int row0) {
-        const int rows[4] = {row0 + 2 * c, row0 + 2 * c + 1, row0 + 8 + 2 * c, row0 + 9 + 2 * c};
+    const int first = begin + warp * 16, stride = kDecWarps * 16;
+    if (lane == 0)
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int hf = 0; hf < HF; ++hf)
-                v[i][hf] = dec_ld16(vbase + (int64_t)rows[i] * D * 2 + hf * 128 + r * 16, rows[i] < end);
-    };
-    if (begin + warp * 16 < end) { load_k(begin + warp * 16); load_v(begin + warp * 16); }
-    for (int row0 = begin + warp * 16; row0 < end; row0 += kDecWarps * 16) {
+        for (int st = 0; st < kDecStages; ++st) issue(first + st * stride, st);
+    int slot = 0;
+    uint32_t parity = 0;
+    bool timed_out = false;
+    for (int row0 = first; row0 < end; row0 += stride) {
         const int vr[4] = {row0 + 2 * c, row0 + 2 * c + 1, row0 + 8 + 2 * c, row0 + 9 + 2 * c};
-        const int next = row0 + kDecWarps * 16;
+        if (!dec_bar_wait(bars + slot, parity)) { timed_out = true; break; }
+        const unsigned char *kblk = ring + (size_t)slot * 2 * kBlockBytes, *vblk = kblk + kBlockBytes;
+        uint4 k1[CH], k2[CH];
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            k1[j] = *reinterpret_cast<const uint4 *>(kblk + r * D * 2 + j * 64 + c * 16);
+            k2[j] = *reinterpret_cast<const uint4 *>(kblk + (8 + r) * D * 2 + j * 64 + c * 16);
+        }
         float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < CH; ++j) {
@@ -197,7 +248,6 @@ decode_mma_kernel(DecArgs a)
             dec_mma(s2, qa[j].x, qb[j].x, qa[j].y, qb[j].y, k2[j].x, k2[j].y);
             dec_mma(s2, qa[j].z, qb[j].z, qa[j].w, qb[j].w, k2[j].z, k2[j].w);
         }
-        if (next < end) load_k(next);
         // lane (r, c): y[hh][0..3] = logits of head r + 8 hh for rows vr[0..3]
         float y[2][4];
 #pragma unroll
@@ -233,6 +283,15 @@ decode_mma_kernel(DecArgs a)
         split_pack(pr[0][2], pr[0][3], ah[2], al[2]);
         split_pack(pr[1][2], pr[1][3], ah[3], al[3]);
         if (!UPPER) ah[1] = ah[3] = al[1] = al[3] = 0u;
+        // rows past the end of a short last block hold what the slot held before: their probabilities
+        // are zero, and zero times a stale NaN must not reach the sums
+        uint4 v[4][HF];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int hf = 0; hf < HF; ++hf)
+                v[i][hf] = vr[i] < end ? *reinterpret_cast<const uint4 *>(vblk + (vr[i] - row0) * D * 2 + hf * 128 + r * 16)
+                                       : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
         for (int hf = 0; hf < HF; ++hf) {
             const uint32_t w0[4] = {v[0][hf].x, v[0][hf].y, v[0][hf].z, v[0][hf].w};
@@ -250,8 +309,15 @@ decode_mma_kernel(DecArgs a)
                     dec_mma(o[t], al[0], al[1], al[2], al[3], b0, b1);
                 }
         }
-        if (next < end) load_v(next);
+        __syncwarp();                                // every lane has read the slot
+        if (lane == 0) issue(row0 + kDecStages * stride, slot);
+        if (++slot == kDecStages) { slot = 0; parity ^= 1u; }
     }
+    if (__any_sync(0xffffffffu, timed_out)) {
+        if (lane == 0 && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_TIMEOUT);
+        for (int st = 0; st < kDecStages; ++st) dec_bar_wait(bars + st, 0) || dec_bar_wait(bars + st, 1);   // let copies in flight land
+    }
+    __syncthreads();                                 // the ring's memory now takes the warps' records
     // the four column lanes of a head hold partial sums of l
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
@@ -427,10 +493,15 @@ cudaError_t run_lanes(const DecArgs &a, dim3 grid, int G, cudaStream_t st)
 template <int D>
 cudaError_t run_mma(const DecArgs &a, dim3 grid, int G, cudaStream_t st)
 {
+    // the staging ring and its barriers; the warps' records reuse the ring's space after the loop
+    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * D * 2 + (size_t)kDecWarps * kDecStages * sizeof(uint64_t);
     if (G <= 8) {
-        decode_mma_kernel<D, false><<<grid, kDecThreads, (size_t)kDecWarps * 8 * (D + 2) * sizeof(float), st>>>(a);
+        const size_t smem = std::max(ring, (size_t)kDecWarps * 8 * (D + 2) * sizeof(float));
+        cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        decode_mma_kernel<D, false><<<grid, kDecThreads, smem, st>>>(a);
     } else {
-        const size_t smem = (size_t)kDecWarps * 16 * (D + 2) * sizeof(float);
+        const size_t smem = std::max(ring, (size_t)kDecWarps * 16 * (D + 2) * sizeof(float));
         cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         decode_mma_kernel<D, true><<<grid, kDecThreads, smem, st>>>(a);

@@ -409,67 +409,46 @@ decode_lanes_kernel(DecArgs a)
     merge_and_store<D>(a, dec_sm, GMAX, G, u, x, nblocks);
 }
 
-// One block per (unit, head): merges the span records and normalises.  The weights 2^(m_b - M)
-// are formed first (a thread per span), then every thread sums its column over a slice of the
-// spans with independent loads; the slices meet in shared memory in slice order.
-constexpr int kCombineThreads = 512;
-constexpr int kMaxSpans = 1024;
-
+// One block per (unit, head), one thread per column: merges the span records in span order and
+// normalises.  Sixteen records are loaded at once (their (max, sum) words are the same for every
+// thread of the block, so the merge weights are simply recomputed by each), so a unit of up to
+// sixteen spans costs one round trip to memory after the offsets.
 template <int D>
-__global__ void __launch_bounds__(kCombineThreads)
+__global__ void __launch_bounds__(D)
 decode_combine_kernel(DecArgs a)
 {
-    constexpr int SL = kCombineThreads / D;         // slices of the span list
-    __shared__ float w[kMaxSpans], wl[kMaxSpans];
-    __shared__ float red[kCombineThreads / 32];
-    __shared__ float acc[SL][D];
-    __shared__ float s_M, s_L;
     const refree_params &p = a.p;
     const int Hkv = p.num_kv_heads, G = p.num_q_heads / Hkv;
     const int u = blockIdx.x / G, h = blockIdx.x % G, s = u / Hkv, g = u % Hkv;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t len64 = a.offsets[u + 1] - a.offsets[u];
     const int len = (int)max((int64_t)0, min(len64, (int64_t)a.span * a.gx));
     const int nblocks = ceil_div(len, a.span);
     if (nblocks <= 1) return;                       // written by the attention kernel itself
     const float *rec0 = a.part + ((int64_t)u * a.gx * G + h) * (D + 2);
     const int64_t stride = (int64_t)G * (D + 2);
-    // M = max of the span maxima
-    float m = -INFINITY;
-    for (int b = tid; b < nblocks; b += kCombineThreads) m = fmaxf(m, rec0[b * stride + D]);
-    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0) red[warp] = m;
-    __syncthreads();
-    if (tid == 0) {
-        float M = -INFINITY;
-        for (int i = 0; i < kCombineThreads / 32; ++i) M = fmaxf(M, red[i]);
-        s_M = M;
-    }
-    __syncthreads();
-    const float M = s_M;
-    for (int b = tid; b < nblocks; b += kCombineThreads) {
-        w[b] = dec_ex2(rec0[b * stride + D] - M);
-        wl[b] = w[b] * rec0[b * stride + D + 1];
-    }
-    __syncthreads();
-    if (tid == 0) {                                 // the denominator, in span order
-        float L = 0.f;
-        for (int b = 0; b < nblocks; ++b) L += wl[b];
-        s_L = L;
-    }
-    const int col = tid % D, sl = tid / D;
-    const int per = ceil_div(nblocks, SL), b0 = sl * per, b1 = min(nblocks, b0 + per);
-    float val = 0.f;
-#pragma unroll 8
-    for (int b = b0; b < b1; ++b) val += w[b] * rec0[b * stride + col];
-    acc[sl][col] = val;
-    __syncthreads();
-    if (tid < D) {
-        float tot = 0.f;
+    float M = -INFINITY, L = 0.f, val = 0.f;
+    for (int b0 = 0; b0 < nblocks; b0 += 16) {
+        float mm[16], ll[16], vv[16];
 #pragma unroll
-        for (int i = 0; i < SL; ++i) tot += acc[i][tid];
-        a.out[((int64_t)s * p.num_q_heads + g * G + h) * D + native_col(tid, a.native)] = s_L > 0.f ? tot / s_L : 0.f;
+        for (int q = 0; q < 16; ++q) {
+            const bool in = b0 + q < nblocks;
+            const float *rec = rec0 + (int64_t)(in ? b0 + q : b0) * stride;
+            mm[q] = in ? __ldcg(rec + D) : -INFINITY;
+            ll[q] = in ? __ldcg(rec + D + 1) : 0.f;
+            vv[q] = in ? __ldcg(rec + threadIdx.x) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const float mn = fmaxf(M, mm[q]);
+            if (mn > -INFINITY) {
+                const float f0 = dec_ex2(M - mn), f1 = dec_ex2(mm[q] - mn);
+                val = val * f0 + vv[q] * f1;
+                L = L * f0 + ll[q] * f1;
+                M = mn;
+            }
+        }
     }
+    a.out[((int64_t)s * p.num_q_heads + g * G + h) * D + native_col(threadIdx.x, a.native)] = L > 0.f ? val / L : 0.f;
 }
 
 template <typename T, int D>
@@ -513,7 +492,7 @@ cudaError_t run_mma(const DecArgs &a, dim3 grid, int G, cudaStream_t st)
 void decode_shape(const refree_params &p, int64_t max_rows, int &gx, int &span)
 {
     const int64_t U = (int64_t)p.num_seqs * p.num_kv_heads;
-    const int64_t want = std::min<int64_t>(kMaxSpans, std::max<int64_t>(1, 148 / U));   // about one block per SM (one wave: prologue and merge are paid once)
+    const int64_t want = std::max<int64_t>(1, 148 / U);   // about one block per SM (one wave: prologue and merge are paid once)
     const int64_t by_rows = std::max<int64_t>(1, (max_rows + 127) / 128);      // at least one 16-row block per warp
     gx = (int)std::min<int64_t>(want, by_rows);
     span = (int)(((max_rows + gx - 1) / gx + 15) / 16 * 16);
@@ -557,8 +536,8 @@ cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, c
     }
     count_launches(1);
     if (e != cudaSuccess || a.gx == 1) return e;
-    if (p.head_dim == 64) decode_combine_kernel<64><<<U * G, kCombineThreads, 0, st>>>(a);
-    else decode_combine_kernel<128><<<U * G, kCombineThreads, 0, st>>>(a);
+    if (p.head_dim == 64) decode_combine_kernel<64><<<U * G, 64, 0, st>>>(a);
+    else decode_combine_kernel<128><<<U * G, 128, 0, st>>>(a);
     count_launches(1);
     return cudaGetLastError();
 }

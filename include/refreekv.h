@@ -158,6 +158,31 @@ refree_status refree_compress_layer_host(const refree_params *p, const void *q_w
                                          int32_t *kept_idx, float *scores,
                                          void *arena, size_t arena_bytes, void *stream);
 
+/* The same host-memory pass for a run of `num_layers` layers that share one
+ * shape (Algorithm 1 is applied layer by layer after prefill, Section 3.3),
+ * pipelined over three internal streams: the inputs of layer l + 1 travel to the
+ * device and the kept rows of layer l - 1 travel back while layer l is compressed,
+ * so the run costs about one direction's copy time per layer.
+ *   q_win, k, v, k_out, v_out, lengths, offsets  arrays of `num_layers` HOST
+ *            pointers, one per layer, each as in refree_compress_layer_host
+ *            (pinned memory lets the copies overlap; pageable memory works but
+ *            serialises them)
+ *   seq_start, seq_len, total_tokens, kv_elems, capacity_rows  common to all layers
+ *   arena    DEVICE buffer of refree_host_pipeline_arena_size() bytes, 256-byte
+ *            aligned: two sets of staging buffers and one workspace
+ * Index lists and scores are not returned (use the per-layer call for them).
+ * The call creates and destroys its streams and events, blocks until every layer
+ * is back in host memory, and returns the first error met (device-side
+ * conditions as REFREE_ERR_CAPACITY / _TIMEOUT / _NONFINITE). */
+refree_status refree_host_pipeline_arena_size(const refree_params *p, int64_t total_tokens, int64_t kv_elems,
+                                              int64_t capacity_rows, size_t *bytes);
+refree_status refree_compress_layers_host(const refree_params *p, int32_t num_layers,
+                                          const void *const *q_win, const void *const *k, const void *const *v,
+                                          int64_t kv_elems, const int32_t *seq_start, const int32_t *seq_len,
+                                          int64_t total_tokens, void *const *k_out, void *const *v_out,
+                                          int64_t capacity_rows, int32_t *const *lengths, int64_t *const *offsets,
+                                          void *arena, size_t arena_bytes);
+
 /* Selection without any device allocation (no counterpart in the paper; the
  * arithmetic and the outputs are exactly those of refree_select_budget).
  *

@@ -89,6 +89,9 @@ SIGNATURES = {
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_host_pipeline_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
+    "refree_compress_layers_host": (ctypes.c_int, [_PP, ctypes.c_int32, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
+                                                   _I64, _VP, _VP, _VP, _SZ]),
     "refree_decode_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
     "refree_decode_attention": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
     "refree_host_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
@@ -253,6 +256,36 @@ def refree_compress_layer_host(p: Params, q_win, k, v, seq_start, seq_len, total
 
 
 # ---- convenience wrapper -----------------------------------------------------
+def refree_host_pipeline_arena_size(p: Params, total_tokens: int, kv_elems: int, capacity_rows: int) -> int:
+    out = _SZ(0)
+    c = p.c_struct()
+    _check(lib().refree_host_pipeline_arena_size(ctypes.byref(c), total_tokens, kv_elems, capacity_rows,
+                                                 ctypes.byref(out)), "refree_host_pipeline_arena_size")
+    return int(out.value)
+
+
+def _ptr_array(tensors):
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t.data_ptr()
+    return arr
+
+
+def refree_compress_layers_host(p: Params, q_win, k, v, seq_start, seq_len, total_tokens, k_out, v_out,
+                                capacity_rows, lengths, offsets, arena, check=True) -> int:
+    """Lists of host tensors, one entry per layer; ``arena`` is a device tensor."""
+    c = p.c_struct()
+    n = len(k)
+    arrays = [_ptr_array(x) for x in (q_win, k, v, k_out, v_out, lengths, offsets)]
+    rc = lib().refree_compress_layers_host(ctypes.byref(c), n, arrays[0], arrays[1], arrays[2], k[0].numel(),
+                                           _dp(seq_start), _dp(seq_len), total_tokens, arrays[3], arrays[4],
+                                           capacity_rows, arrays[5], arrays[6], _dp(arena),
+                                           arena.numel() * arena.element_size())
+    if check:
+        _check(rc, "refree_compress_layers_host")
+    return rc
+
+
 @dataclasses.dataclass
 class LayerResult:
     k_out: torch.Tensor

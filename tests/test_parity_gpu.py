@@ -222,6 +222,38 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert torch.equal(scores, dev_res.scores.cpu())
 
 
+@pytest.mark.parametrize("rank_mode", [binding.RANK_POSITION, binding.RANK_SCORE])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_pipelined_host_run_of_layers_matches_the_per_layer_call(rank_mode, pinned):
+    # five layers through the three-stream pipeline (two staging slots, so slots are reused twice)
+    cfg = small_cfg(window=16, dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2)
+    n_layers = 5
+    lays = [workloads.make_layer(cfg, l, seq_lens=[700, 90, 333]) for l in range(n_layers)]
+    p = binding.params_for(cfg, lays[0], rank_mode=rank_mode, threshold=0.05)
+    total = lays[0].total_tokens
+    cap = p.num_kv_heads * total
+    units = p.num_seqs * p.num_kv_heads
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    q = [pin(l.q_win) for l in lays]
+    k = [pin(l.k) for l in lays]
+    v = [pin(l.v) for l in lays]
+    k_out = [pin(torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype)) for _ in lays]
+    v_out = [pin(torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype)) for _ in lays]
+    lengths = [torch.zeros(units, dtype=torch.int32) for _ in lays]
+    offsets = [torch.zeros(units + 1, dtype=torch.int64) for _ in lays]
+    arena = torch.empty(binding.refree_host_pipeline_arena_size(p, total, lays[0].k.numel(), cap), dtype=torch.uint8,
+                        device=DEV)
+    binding.refree_compress_layers_host(p, q, k, v, lays[0].seq_start, lays[0].seq_len, total, k_out, v_out, cap,
+                                        lengths, offsets, arena)
+    for l, lay in enumerate(lays):
+        ref = binding.compress_layer(p, *_device_inputs(lay), total, want_scores=False, want_kept_idx=False)
+        torch.cuda.synchronize()
+        rows = int(offsets[l][-1])
+        assert torch.equal(lengths[l], ref.lengths.cpu().reshape(-1)) and torch.equal(offsets[l], ref.offsets.cpu())
+        assert torch.equal(parity.bits(k_out[l][:rows]), parity.bits(ref.k_out[:rows].cpu()))
+        assert torch.equal(parity.bits(v_out[l][:rows]), parity.bits(ref.v_out[:rows].cpu()))
+
+
 @pytest.mark.parametrize("dtype,d,hq,hkv", [("bf16", 128, 28, 4), ("fp32", 64, 4, 2), ("bf16", 64, 16, 1), ("fp32", 128, 3, 3)])
 @pytest.mark.parametrize("rank_mode,scope", [(binding.RANK_POSITION, binding.SCOPE_HEAD),
                                              (binding.RANK_SCORE, binding.SCOPE_HEAD),

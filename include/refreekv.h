@@ -138,6 +138,35 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
                                     void *workspace, size_t workspace_bytes,
                                     int32_t *device_status, void *stream);
 
+/* The pass of Algorithm 1 for a run of `num_layers` device-resident layers that
+ * share one shape (Section 3.3: the cache of every layer is compressed once,
+ * after prefill).  Scoring is bound by the tensor pipes and compaction by HBM,
+ * so the run is software-pipelined over two internal streams: layer l + 1 is
+ * scored and its budgets chosen while the kept rows of layer l are copied.
+ * Results are bit-identical to num_layers calls of refree_compress_layer.
+ *   q_win, k, v, k_out, v_out, lengths, offsets  HOST arrays of `num_layers`
+ *            DEVICE pointers, one per layer, each as in refree_compress_layer;
+ *            the arrays themselves are read before the call returns
+ *   seq_start, seq_len, total_tokens, capacity_rows  common to all layers (device
+ *            pointers as in refree_compress_layer)
+ *   workspace  refree_layers_workspace_size() bytes (two per-layer workspaces),
+ *            256-byte aligned, device
+ * Index lists and scores are not returned (use the per-layer call for them).
+ * Nothing is allocated in device memory and the host is not synchronised: the
+ * work is ordered after what `stream` holds at the call, and `stream` continues
+ * only when every layer is done.  The first call on a device creates the two
+ * internal streams (highest priority for scoring, lowest for compaction) and
+ * their events, which live until the process exits; calls from several host
+ * threads on one device share them and are serialised by stream order. */
+refree_status refree_layers_workspace_size(const refree_params *p, int64_t total_tokens, size_t *bytes);
+refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
+                                     const void *const *q_win, const void *const *k, const void *const *v,
+                                     const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                                     void *const *k_out, void *const *v_out, int64_t capacity_rows,
+                                     int32_t *const *lengths, int64_t *const *offsets,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *device_status, void *stream);
+
 /* The same pass of Algorithm 1 for callers whose cache lives in HOST memory
  * (pinned or pageable): q_win, k, v, seq_start, seq_len are host pointers, and
  * so are the outputs k_out, v_out (capacity_rows rows), lengths, offsets,

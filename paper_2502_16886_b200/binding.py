@@ -89,6 +89,9 @@ SIGNATURES = {
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_layers_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
+    "refree_compress_layers": (ctypes.c_int, [_PP, ctypes.c_int32, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64,
+                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
     "refree_host_pipeline_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
     "refree_compress_layers_host": (ctypes.c_int, [_PP, ctypes.c_int32, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                                    _I64, _VP, _VP, _VP, _SZ]),
@@ -283,6 +286,37 @@ def refree_compress_layers_host(p: Params, q_win, k, v, seq_start, seq_len, tota
                                            arena.numel() * arena.element_size())
     if check:
         _check(rc, "refree_compress_layers_host")
+    return rc
+
+
+def refree_layers_workspace_size(p: Params, total_tokens: int) -> int:
+    out = _SZ(0)
+    c = p.c_struct()
+    _check(lib().refree_layers_workspace_size(ctypes.byref(c), total_tokens, ctypes.byref(out)),
+           "refree_layers_workspace_size")
+    return int(out.value)
+
+
+class LayerPointers:
+    """The seven per-layer pointer arrays of ``refree_compress_layers``, built once for lists of device
+    tensors (one entry per layer) so that repeated calls marshal nothing."""
+
+    def __init__(self, q_win, k, v, k_out, v_out, lengths, offsets):
+        self.num_layers = len(k)
+        self.keep = (q_win, k, v, k_out, v_out, lengths, offsets)
+        self.arrays = [_ptr_array(x) for x in self.keep]
+
+
+def refree_compress_layers(p: Params, ptrs: LayerPointers, seq_start, seq_len, total_tokens, capacity_rows,
+                           workspace, device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    a = ptrs.arrays
+    rc = lib().refree_compress_layers(ctypes.byref(c), ptrs.num_layers, a[0], a[1], a[2], _dp(seq_start), _dp(seq_len),
+                                      total_tokens, a[3], a[4], capacity_rows, a[5], a[6], _dp(workspace),
+                                      workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                      _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compress_layers")
     return rc
 
 

@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <mutex>
 
 #include "refree_internal.cuh"
 
@@ -232,6 +233,44 @@ refree_status refree_decode_attention(const refree_params *p, const void *q_new,
                                              device_status, (cudaStream_t)stream));
 }
 
+// The launch sequence of one layer.  `cs` takes scoring and selection; compaction goes to `cc`
+// (after `scored`, recorded on `cs`, when the two differ).
+static refree_status enqueue_layer(const refree_params *p, const void *q_win, const void *k, const void *v,
+                                   const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                                   void *k_out, void *v_out, int64_t capacity_rows, int32_t *lengths,
+                                   int64_t *offsets, int32_t *kept_idx, float *scores, char *ws,
+                                   const Workspace &lay, int32_t *device_status, cudaStream_t cs,
+                                   cudaStream_t cc, cudaEvent_t scored)
+{
+    float *sc = scores ? scores : reinterpret_cast<float *>(ws + lay.scores_off);
+    const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
+    int32_t *kept = kept_idx ? kept_idx : (ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off));
+    cudaError_t e = cudaSuccess;
+    // a frozen layer needs no scores unless the caller asked for them
+    // position ranking per head on the tensor-core path: the scoring kernel also leaves the per-32-position
+    // sums of squares, and the stopping rule reads those instead of every score
+    GroupPartial *groups = nullptr;
+    if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
+        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
+        groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
+    if (total_tokens > 0 && (!p->force_full || scores))
+        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    // with two-range kept sets and no index list wanted, the compaction kernel forms the offsets itself
+    const bool lean = ranges && !kept;
+    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs,
+                      !lean, groups);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    const bool split = cc != cs;
+    if (split) {
+        if (cudaEventRecord(scored, cs) != cudaSuccess || cudaStreamWaitEvent(cc, scored, 0) != cudaSuccess)
+            return REFREE_ERR_CUDA;
+    }
+    e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, lean ? offsets : nullptr, k_out,
+                       v_out, capacity_rows, device_status, cc, split && use_tc(*p, q_win));
+    return from_cuda(e);
+}
+
 refree_status refree_compress_layer(const refree_params *p, const void *q_win,
                                     const void *k, const void *v,
                                     const int32_t *seq_start, const int32_t *seq_len,
@@ -254,30 +293,100 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
     const Workspace lay = workspace_layout(*p, total_tokens);
     if (!workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
         return REFREE_ERR_WORKSPACE;
-    char *ws = (char *)workspace;
     cudaStream_t cs = (cudaStream_t)stream;
-    float *sc = scores ? scores : reinterpret_cast<float *>(ws + lay.scores_off);
-    const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
-    int32_t *kept = kept_idx ? kept_idx : (ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off));
-    cudaError_t e = cudaSuccess;
-    // a frozen layer needs no scores unless the caller asked for them
-    // position ranking per head on the tensor-core path: the scoring kernel also leaves the per-32-position
-    // sums of squares, and the stopping rule reads those instead of every score
-    GroupPartial *groups = nullptr;
-    if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
-        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
-        groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
-    if (total_tokens > 0 && (!p->force_full || scores))
-        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);
-    if (e != cudaSuccess) return REFREE_ERR_CUDA;
-    // with two-range kept sets and no index list wanted, the compaction kernel forms the offsets itself
-    const bool lean = ranges && !kept;
-    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, capacity_rows, ws, lay, device_status, cs,
-                      !lean, groups);
-    if (e != cudaSuccess) return REFREE_ERR_CUDA;
-    e = launch_compact(*p, k, v, seq_start, seq_len, lengths, offsets, kept, ranges, lean ? offsets : nullptr, k_out,
-                       v_out, capacity_rows, device_status, cs);
-    return from_cuda(e);
+    return enqueue_layer(p, q_win, k, v, seq_start, seq_len, total_tokens, k_out, v_out, capacity_rows, lengths,
+                         offsets, kept_idx, scores, (char *)workspace, lay, device_status, cs, cs, nullptr);
+}
+
+// ---- a run of device-resident layers, compaction of layer l under the scoring of layer l + 1 ----
+namespace {
+struct LayerPipe {
+    bool ready = false;
+    cudaStream_t hi = nullptr, lo = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, scored[2] = {nullptr, nullptr}, compacted[2] = {nullptr, nullptr};
+};
+std::mutex g_pipe_mutex;
+LayerPipe g_pipe[64];
+
+// Streams and events of the current device, made on first use and kept until the process exits.
+LayerPipe *layer_pipe()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    LayerPipe &lp = g_pipe[dev];
+    if (lp.ready) return &lp;
+    int least = 0, greatest = 0;
+    if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) return nullptr;
+    bool ok = cudaStreamCreateWithPriority(&lp.hi, cudaStreamNonBlocking, greatest) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&lp.lo, cudaStreamNonBlocking, least) == cudaSuccess &&
+              cudaEventCreateWithFlags(&lp.fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&lp.join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+        ok = cudaEventCreateWithFlags(&lp.scored[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&lp.compacted[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    lp.ready = true;
+    return &lp;
+}
+}  // namespace
+
+refree_status refree_layers_workspace_size(const refree_params *p, int64_t total_tokens, size_t *bytes)
+{
+    const refree_status st = refree_workspace_size(p, total_tokens, bytes);
+    if (st == REFREE_OK) *bytes *= 2;
+    return st;
+}
+
+refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
+                                     const void *const *q_win, const void *const *k, const void *const *v,
+                                     const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                                     void *const *k_out, void *const *v_out, int64_t capacity_rows,
+                                     int32_t *const *lengths, int64_t *const *offsets,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    if (num_layers < 0 || !q_win || !k || !v || !seq_start || !seq_len || !k_out || !v_out || !lengths || !offsets ||
+        capacity_rows < 0)
+        return REFREE_ERR_INVALID_ARG;
+    for (int l = 0; l < num_layers; ++l) {
+        if (!q_win[l] || !k[l] || !v[l] || !k_out[l] || !v_out[l] || !lengths[l] || !offsets[l])
+            return REFREE_ERR_INVALID_ARG;
+        st = check_kv_layout(p, k[l], v[l], true);
+        if (st != REFREE_OK) return st;
+        if ((reinterpret_cast<uintptr_t>(k_out[l]) & 15) || (reinterpret_cast<uintptr_t>(v_out[l]) & 15))
+            return REFREE_ERR_UNSUPPORTED;
+    }
+    const Workspace lay = workspace_layout(*p, total_tokens);
+    if (!workspace || workspace_bytes < 2 * lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    if (num_layers == 0) return REFREE_OK;
+    LayerPipe *lp = layer_pipe();
+    if (!lp) return REFREE_ERR_CUDA;
+    cudaStream_t cs = (cudaStream_t)stream;
+    bool ok = cudaEventRecord(lp->fork, cs) == cudaSuccess && cudaStreamWaitEvent(lp->hi, lp->fork, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(lp->lo, lp->fork, 0) == cudaSuccess;
+    refree_status result = ok ? REFREE_OK : REFREE_ERR_CUDA;
+    for (int l = 0; l < num_layers && result == REFREE_OK; ++l) {
+        const int slot = l & 1;
+        // the half of the workspace is free once the compaction of layer l - 2 has read its budgets
+        if (l >= 2 && cudaStreamWaitEvent(lp->hi, lp->compacted[slot], 0) != cudaSuccess) { result = REFREE_ERR_CUDA; break; }
+        result = enqueue_layer(p, q_win[l], k[l], v[l], seq_start, seq_len, total_tokens, k_out[l], v_out[l],
+                               capacity_rows, lengths[l], offsets[l], nullptr, nullptr,
+                               (char *)workspace + (size_t)slot * lay.total, lay, device_status, lp->hi, lp->lo,
+                               lp->scored[slot]);
+        if (result != REFREE_OK) break;
+        if (cudaEventRecord(lp->compacted[slot], lp->lo) != cudaSuccess) { result = REFREE_ERR_CUDA; break; }
+    }
+    // the caller's stream continues after everything that was enqueued, whatever happened
+    if (ok) {
+        if (cudaEventRecord(lp->join, lp->hi) != cudaSuccess || cudaStreamWaitEvent(cs, lp->join, 0) != cudaSuccess ||
+            cudaEventRecord(lp->join, lp->lo) != cudaSuccess || cudaStreamWaitEvent(cs, lp->join, 0) != cudaSuccess)
+            if (result == REFREE_OK) result = REFREE_ERR_CUDA;
+    }
+    return result;
 }
 
 refree_status refree_host_arena_size(const refree_params *p, int64_t total_tokens,

@@ -9,6 +9,7 @@ namespace refree {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kThreadsSlim = 128;   // block that fits beside a resident scoring CTA (see launch_compact)
 constexpr int kUnroll = 4;
 
 __device__ inline int4 ld_stream(const int4 *p)
@@ -24,6 +25,7 @@ __device__ inline void st_stream(int4 *p, const int4 &v)
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+template <int kThreads>
 __global__ void __launch_bounds__(kThreads)
 compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq_start,
                const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
@@ -98,11 +100,23 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            const int32_t *seq_start, const int32_t *seq_len,
                            const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
                            bool position_ranges, int64_t *offsets_out, void *k_out, void *v_out,
-                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st)
+                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st, bool beside_scoring)
 {
     const int U = p.num_seqs * p.num_kv_heads;
+    if (beside_scoring) {
+        // The launch shares the SMs with a persistent scoring CTA of the next layer (576 threads, 96
+        // registers each): 10 240 registers are left per SM, so the block is 128 threads (8 192
+        // registers), and the grid is many short-lived blocks, so that a scoring CTA that becomes
+        // runnable finds room as soon as a few of them retire.
+        const int gx = max(1, (148 * 32) / U);
+        compact_kernel<kThreadsSlim><<<dim3(gx, U), kThreadsSlim, 0, st>>>(
+            p, (const char *)k, (const char *)v, seq_start, seq_len, lengths, offsets, kept_idx,
+            position_ranges ? 1 : 0, offsets_out, (char *)k_out, (char *)v_out, capacity_rows, dev_status);
+        count_launches(1);
+        return cudaGetLastError();
+    }
     const int gx = max(1, (148 * 8) / U);
-    compact_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
+    compact_kernel<kThreads><<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
                                                      lengths, offsets, kept_idx, position_ranges ? 1 : 0, offsets_out,
                                                      (char *)k_out, (char *)v_out, capacity_rows, dev_status);
     count_launches(1);

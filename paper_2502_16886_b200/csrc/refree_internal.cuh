@@ -149,7 +149,8 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            const int32_t *seq_start, const int32_t *seq_len,
                            const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
                            bool position_ranges, int64_t *offsets_out, void *k_out, void *v_out,
-                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st);
+                           int64_t capacity_rows, int32_t *dev_status, cudaStream_t st,
+                           bool beside_scoring = false);
 
 size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,

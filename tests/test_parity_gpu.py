@@ -254,6 +254,60 @@ def test_pipelined_host_run_of_layers_matches_the_per_layer_call(rank_mode, pinn
         assert torch.equal(parity.bits(v_out[l][:rows]), parity.bits(ref.v_out[:rows].cpu()))
 
 
+@pytest.mark.parametrize("rank_mode,window,dtype", [(binding.RANK_POSITION, 16, "bf16"), (binding.RANK_SCORE, 16, "bf16"),
+                                                    (binding.RANK_POSITION, 1, "bf16"), (binding.RANK_POSITION, 8, "fp32")])
+def test_pipelined_device_run_of_layers_matches_the_per_layer_call(rank_mode, window, dtype):
+    """refree_compress_layers (scoring of layer l + 1 over the compaction of layer l, two internal
+    streams, two workspace halves) against one refree_compress_layer call per layer: five layers, so
+    each half is reused, twice in a row on the same buffers, then once more after other work on the
+    caller's stream."""
+    cfg = small_cfg(window=window, dtype=dtype, head_dim=128, num_q_heads=8, num_kv_heads=2)
+    n_layers = 5
+    lays = [workloads.make_layer(cfg, l, seq_lens=[2700, 90, 1333]) for l in range(n_layers)]
+    p = binding.params_for(cfg, lays[0], rank_mode=rank_mode, threshold=0.05)
+    total = lays[0].total_tokens
+    cap = p.num_kv_heads * total
+    units = p.num_seqs * p.num_kv_heads
+    dev_in = [_device_inputs(l) for l in lays]
+    refs = [binding.compress_layer(p, *d, total, want_scores=False, want_kept_idx=False) for d in dev_in]
+    torch.cuda.synchronize()
+    k_out = [torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype, device=DEV) for _ in lays]
+    v_out = [torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype, device=DEV) for _ in lays]
+    lengths = [torch.zeros(units, dtype=torch.int32, device=DEV) for _ in lays]
+    offsets = [torch.zeros(units + 1, dtype=torch.int64, device=DEV) for _ in lays]
+    ptrs = binding.LayerPointers([d[0] for d in dev_in], [d[1] for d in dev_in], [d[2] for d in dev_in], k_out, v_out,
+                                 lengths, offsets)
+    ws = torch.empty(binding.refree_layers_workspace_size(p, total), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for rep in range(3):
+        for t in k_out + v_out + lengths + offsets:
+            t.fill_(0 if rep != 1 else 1)              # ordered before the run on the caller's stream
+        binding.refree_compress_layers(p, ptrs, dev_in[0][3], dev_in[0][4], total, cap, ws, status)
+        got = [(ln.clone(), of.clone(), ko.clone(), vo.clone()) for ln, of, ko, vo in zip(lengths, offsets, k_out, v_out)]
+        torch.cuda.synchronize()                       # the clones were ordered after the run by the join
+        assert status.item() == 0
+        for l, ref in enumerate(refs):
+            ln, of, ko, vo = got[l]
+            rows = int(of[-1])
+            assert rows == int(ref.offsets[-1]) and 0 < rows <= cap
+            assert torch.equal(ln, ref.lengths.reshape(-1)) and torch.equal(of, ref.offsets)
+            assert torch.equal(parity.bits(ko[:rows]), parity.bits(ref.k_out[:rows]))
+            assert torch.equal(parity.bits(vo[:rows]), parity.bits(ref.v_out[:rows]))
+
+
+def test_pipelined_device_run_rejects_a_single_workspace():
+    cfg = small_cfg(window=16, dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[300])
+    p = binding.params_for(cfg, lay)
+    d = _device_inputs(lay)
+    cap = p.num_kv_heads * 300
+    outs = [torch.zeros(cap, 128, dtype=lay.k.dtype, device=DEV) for _ in range(2)]
+    ln, of = torch.zeros(2, dtype=torch.int32, device=DEV), torch.zeros(3, dtype=torch.int64, device=DEV)
+    ptrs = binding.LayerPointers([d[0]], [d[1]], [d[2]], [outs[0]], [outs[1]], [ln], [of])
+    ws = torch.empty(binding.refree_workspace_size(p, 300), dtype=torch.uint8, device=DEV)
+    assert binding.refree_compress_layers(p, ptrs, d[3], d[4], 300, cap, ws, check=False) == binding.ERR_WORKSPACE
+
+
 @pytest.mark.parametrize("dtype,d,hq,hkv", [("bf16", 128, 28, 4), ("fp32", 64, 4, 2), ("bf16", 64, 16, 1), ("fp32", 128, 3, 3)])
 @pytest.mark.parametrize("rank_mode,scope", [(binding.RANK_POSITION, binding.SCOPE_HEAD),
                                              (binding.RANK_SCORE, binding.SCOPE_HEAD),

@@ -375,6 +375,33 @@ def run_ours(args):
                    "bytes_per_layer": int(dec_bytes), "achieved": round(dec_gbs, 1), "peak": peak,
                    "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(dec_gbs / peak, 4)}
 
+    # in-place form of the compaction stage; it overwrites the synthetic cache, so it runs after every other
+    # device sweep (a repeat moves the same rows again: same budgets, same traffic)
+    def inplace(d):
+        binding.refree_compact_inplace(params, d["k"], d["v"], seq_start, seq_len, d["offsets"],
+                                       None if rank_mode == binding.RANK_POSITION else kept, status)
+
+    if rank_mode == binding.RANK_POSITION:
+        for d in layers:
+            inplace(d)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for d in layers:
+                inplace(d)
+        e1.record()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, f"device status {int(status.item())}"
+        inp_ms = e0.elapsed_time(e1) / (reps * L)
+        inplace_line = {"kernel": "refree_compact_inplace", "bound": "hbm", "ms_per_layer": round(inp_ms, 5),
+                        "bytes_per_layer": int(stage_bytes["compact"]),
+                        "achieved": round(stage_bytes["compact"] / (inp_ms * 1e-3) / 1e9, 1), "peak": peak,
+                        "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                        "frac": round(stage_bytes["compact"] / (inp_ms * 1e-3) / 1e9 / peak, 4)}
+    else:
+        inplace_line = None
+
     e2e = measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args)
     cpu_baseline = measure_cpu_baseline(cfg, rank_mode, total, args) if world == 1 and not args.no_cpu_baseline else None
 
@@ -391,6 +418,7 @@ def run_ours(args):
                    "replicas": world},
         "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
         "roofline": roofline, "roofline_pass": roofline_pass, "decode_attention": decode_line,
+        "compact_inplace": inplace_line,
         "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line), flush=True)

@@ -87,6 +87,7 @@ SIGNATURES = {
     "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
     "refree_select_budget_static": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
+    "refree_compact_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
     "refree_layers_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
@@ -199,6 +200,17 @@ def refree_compact(p: Params, k, v, seq_start, seq_len, lengths, offsets, kept_i
                               _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_compact")
+    return rc
+
+
+def refree_compact_inplace(p: Params, k, v, seq_start, seq_len, offsets, kept_idx, device_status=None, stream=None,
+                           check=True) -> int:
+    """Slides every unit's kept rows to the front of its own region of ``k`` and ``v``."""
+    c = p.c_struct()
+    rc = lib().refree_compact_inplace(ctypes.byref(c), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len), _dp(offsets),
+                                      _dp(kept_idx), _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compact_inplace")
     return rc
 
 

@@ -3,6 +3,10 @@
 // loads and stores, several rows in flight per thread.  Rows are copied bit for
 // bit.  With position ranking the kept set is two contiguous ranges, so the
 // source row follows from (b, m, n) and no index list is read.
+#include <cooperative_groups.h>
+
+#include <algorithm>
+
 #include "refree_internal.cuh"
 
 namespace refree {
@@ -94,6 +98,77 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
     }
 }
 
+
+// In-place form of the same step.  Every kept row moves towards the front of its own unit
+// (destination index t <= source index), so rows can be overwritten as soon as whoever
+// needs their old contents has read them.  The kept rows of all units, in order, are cut
+// into rounds of as many 16-byte pieces as the grid holds in registers; in a round every
+// thread loads its pieces, the grid synchronises, and every thread stores them.  A round
+// reads only rows at or beyond its own destinations, which lie beyond every destination of
+// the rounds before it, so one grid barrier per round is all the ordering needed.
+constexpr int kUnrollInplace = 4;
+
+__global__ void __launch_bounds__(kThreads)
+compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_start, const int32_t *seq_len,
+                       const int64_t *offsets, const int32_t *kept_idx, int position_ranges, int32_t *dev_status)
+{
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    const int Hkv = p.num_kv_heads, U = p.num_seqs * Hkv;
+    const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const int vec_per_row = (p.head_dim * esz) >> 4;
+    const int vshift = 31 - __clz(vec_per_row);
+    const int64_t total_vec = max((long long)__ldg(offsets + U), 0ll) << vshift;
+    const int64_t lanes = (int64_t)gridDim.x * kThreads;
+    const int64_t per_round = lanes * kUnrollInplace;
+    const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
+    bool bad = false;
+    for (int64_t base = 0; base < total_vec; base += per_round) {     // the same trip count in every thread
+        int4 kv[kUnrollInplace], vv[kUnrollInplace];
+        char *kd[kUnrollInplace], *vd[kUnrollInplace];
+#pragma unroll
+        for (int r = 0; r < kUnrollInplace; ++r) {
+            kd[r] = vd[r] = nullptr;
+            const int64_t e = base + r * lanes + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+            if (e >= total_vec) continue;
+            const int64_t row = e >> vshift;
+            const int c = (int)(e & (vec_per_row - 1));
+            int lo = 0, hi = U;                                       // unit whose rows contain `row`
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (__ldg(offsets + mid) <= row) lo = mid; else hi = mid;
+            }
+            const int u = lo, s = u / Hkv, g = u % Hkv;
+            const int64_t off = __ldg(offsets + u);
+            const int n = max(__ldg(seq_len + s), 0);
+            const int64_t b64 = __ldg(offsets + u + 1) - off;
+            const int t = (int)(row - off);
+            if (off < 0 || b64 < 0 || b64 > n) { bad = true; continue; }
+            const int b = (int)b64;
+            const int head = min(b, min(p.sink, n));
+            const int src = position_ranges ? (t < head ? t : n - b + t) : __ldg(kept_idx + row);
+            if (src < t || src >= n) { bad = true; continue; }
+            if (src == t) continue;                                   // already in place
+            const int64_t tok0 = __ldg(seq_start + s);
+            char *kb = k + ((int64_t)s * p.k_stride_seq + tok0 * p.k_stride_tok + (int64_t)g * p.k_stride_head) * esz + c * 16;
+            char *vb = v + ((int64_t)s * p.v_stride_seq + tok0 * p.v_stride_tok + (int64_t)g * p.v_stride_head) * esz + c * 16;
+            kv[r] = __ldcg(reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok));
+            vv[r] = __ldcg(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok));
+            kd[r] = kb + (int64_t)t * k_tok;
+            vd[r] = vb + (int64_t)t * v_tok;
+        }
+        grid.sync();
+#pragma unroll
+        for (int r = 0; r < kUnrollInplace; ++r) {
+            if (kd[r]) {
+                *reinterpret_cast<int4 *>(kd[r]) = kv[r];
+                *reinterpret_cast<int4 *>(vd[r]) = vv[r];
+            }
+        }
+    }
+    if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
+}
+
 }  // namespace
 
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
@@ -119,6 +194,36 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
     compact_kernel<kThreads><<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
                                                      lengths, offsets, kept_idx, position_ranges ? 1 : 0, offsets_out,
                                                      (char *)k_out, (char *)v_out, capacity_rows, dev_status);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, const int32_t *seq_start,
+                                   const int32_t *seq_len, const int64_t *offsets, const int32_t *kept_idx,
+                                   bool position_ranges, int32_t *dev_status, cudaStream_t st)
+{
+    static int grid_blocks[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (grid_blocks[dev] == 0) {
+        // every block of the grid must be resident at once: the rounds end in a grid-wide barrier
+        int sms = 0, per_sm = 0, coop = 0;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) != cudaSuccess) return e;
+        if (!coop) return cudaErrorNotSupported;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compact_inplace_kernel, kThreads, 0)) != cudaSuccess)
+            return e;
+        if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+        grid_blocks[dev] = sms * std::min(per_sm, 4);
+    }
+    refree_params pv = p;
+    char *kc = (char *)k, *vc = (char *)v;
+    int ranges = position_ranges ? 1 : 0;
+    void *args[9] = {&pv, &kc, &vc, &seq_start, &seq_len, &offsets, &kept_idx, &ranges, &dev_status};
+    e = cudaLaunchCooperativeKernel((const void *)compact_inplace_kernel, dim3(grid_blocks[dev]), dim3(kThreads), args, 0, st);
+    if (e != cudaSuccess) return e;
     count_launches(1);
     return cudaGetLastError();
 }

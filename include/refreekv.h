@@ -125,28 +125,39 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
                              int64_t capacity_rows, int32_t *device_status, void *stream);
 
 /* Step S7 in place, for callers with no room for a second copy of the cache.
- * Position ranking (Section 3.2 "Initial Ranking") keeps the leading positions
- * and a suffix, so the leading rows stay where they are and the suffix slides
- * down behind them; with score ranking the kept rows (ascending kept_idx) slide
- * down the same way.  Afterwards the first b = offsets[u+1] - offsets[u] rows of
- * every unit's OWN region of K and V hold its compacted cache, bit for bit the
- * rows refree_compact would have written to k_out / v_out:
- *     K[s, t, g, :] <- K[s, kept(u, t), g, :]   for t < b   (same strides as the input)
- * Rows at and beyond b keep stale contents.  The cache stays a strided ragged
- * array addressed by (seq_start, strides, per-unit length); it is not the dense
- * [sum b, head_dim] array that refree_decode_attention reads.
+ * The kept rows of every unit end up contiguous inside the unit's OWN region of
+ * K and V (same strides as the input), bit for bit the rows refree_compact would
+ * have written to k_out / v_out, in the same order.  With b = offsets[u+1] -
+ * offsets[u] and n the sequence length:
+ *   REFREE_ANCHOR_FRONT  rows [0, b) of the unit hold its compacted cache:
+ *       K[s, t, g, :] <- K[s, kept(u, t), g, :] for t < b.  Position ranking
+ *       (Section 3.2 "Initial Ranking") keeps the leading positions and a suffix,
+ *       so the leading rows stay and the suffix slides down behind them; with
+ *       score ranking the kept rows (ascending kept_idx) slide down the same way.
+ *       Every kept row is read and written once.
+ *   REFREE_ANCHOR_BACK   rows [n - b, n) of the unit hold its compacted cache.
+ *       Position ranking (or force_full) only: the suffix is already in place, so
+ *       only the leading rows (at most `sink` per unit) are lifted to just below
+ *       it - a few KB per unit instead of the whole kept cache - and rows that
+ *       decoding appends at n, n + 1, .. stay contiguous with it.  Score ranking
+ *       returns REFREE_ERR_UNSUPPORTED.
+ * Rows outside the stated range keep stale contents.  The cache stays a strided
+ * ragged array addressed by (seq_start, strides, per-unit length); it is not the
+ * dense [sum b, head_dim] array that refree_decode_attention reads.
  *   k, v      device, read and written
  *   offsets   [num_seqs*num_kv_heads + 1] int64, as produced by refree_select_budget
  *   kept_idx  as produced by refree_select_budget; ignored (may be null) with
  *             position ranking or force_full, required with score ranking
- * Uses no scratch memory.  The kernel ends each round of copies with a grid-wide
- * barrier and is therefore launched cooperatively (all its blocks resident);
- * REFREE_ERR_CUDA is returned where the device cannot do that.  Budgets outside
- * [0, n] or sources outside [t, n) set REFREE_DEV_CAPACITY in *device_status and
- * those pieces are skipped. */
+ * Uses no scratch memory.  The FRONT kernel ends each round of copies with a
+ * grid-wide barrier and is therefore launched cooperatively (all its blocks
+ * resident); REFREE_ERR_CUDA is returned where the device cannot do that.
+ * Budgets outside [0, n] or sources outside [t, n) set REFREE_DEV_CAPACITY in
+ * *device_status and those pieces are skipped. */
+#define REFREE_ANCHOR_FRONT 0
+#define REFREE_ANCHOR_BACK 1
 refree_status refree_compact_inplace(const refree_params *p, void *k, void *v,
                                      const int32_t *seq_start, const int32_t *seq_len,
-                                     const int64_t *offsets, const int32_t *kept_idx,
+                                     const int64_t *offsets, const int32_t *kept_idx, int32_t anchor,
                                      int32_t *device_status, void *stream);
 
 /* The whole per-layer pass of Algorithm 1 (everything after the prefill of the

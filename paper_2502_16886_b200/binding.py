@@ -24,6 +24,7 @@ DEV_CAPACITY, DEV_TIMEOUT, DEV_NONFINITE = 1, 2, 4
 RANK_POSITION, RANK_SCORE = 0, 1
 SCOPE_HEAD, SCOPE_LAYER = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
+ANCHOR_FRONT, ANCHOR_BACK = 0, 1
 
 
 class RefreeError(RuntimeError):
@@ -87,7 +88,7 @@ SIGNATURES = {
     "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
     "refree_select_budget_static": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
-    "refree_compact_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP]),
+    "refree_compact_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
     "refree_layers_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
@@ -204,11 +205,11 @@ def refree_compact(p: Params, k, v, seq_start, seq_len, lengths, offsets, kept_i
 
 
 def refree_compact_inplace(p: Params, k, v, seq_start, seq_len, offsets, kept_idx, device_status=None, stream=None,
-                           check=True) -> int:
-    """Slides every unit's kept rows to the front of its own region of ``k`` and ``v``."""
+                           check=True, anchor=ANCHOR_FRONT) -> int:
+    """Gathers every unit's kept rows at the front (or, ``ANCHOR_BACK``, the end) of its own region of ``k`` and ``v``."""
     c = p.c_struct()
     rc = lib().refree_compact_inplace(ctypes.byref(c), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len), _dp(offsets),
-                                      _dp(kept_idx), _dp(device_status), _stream(stream))
+                                      _dp(kept_idx), anchor, _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_compact_inplace")
     return rc

@@ -196,18 +196,20 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
 
 refree_status refree_compact_inplace(const refree_params *p, void *k, void *v,
                                      const int32_t *seq_start, const int32_t *seq_len,
-                                     const int64_t *offsets, const int32_t *kept_idx,
+                                     const int64_t *offsets, const int32_t *kept_idx, int32_t anchor,
                                      int32_t *device_status, void *stream)
 {
     refree_status st = check_params(p, 0);
     if (st != REFREE_OK) return st;
     if (!k || !v || !seq_start || !seq_len || !offsets) return REFREE_ERR_INVALID_ARG;
+    if (anchor != REFREE_ANCHOR_FRONT && anchor != REFREE_ANCHOR_BACK) return REFREE_ERR_INVALID_ARG;
     const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
     if (!ranges && !kept_idx) return REFREE_ERR_INVALID_ARG;
+    if (!ranges && anchor == REFREE_ANCHOR_BACK) return REFREE_ERR_UNSUPPORTED;
     st = check_kv_layout(p, k, v, true);
     if (st != REFREE_OK) return st;
     return from_cuda(launch_compact_inplace(*p, k, v, seq_start, seq_len, offsets, ranges ? nullptr : kept_idx, ranges,
-                                            device_status, (cudaStream_t)stream));
+                                            anchor == REFREE_ANCHOR_BACK, device_status, (cudaStream_t)stream));
 }
 
 static refree_status check_decode(const refree_params *p, int64_t max_rows)

@@ -169,6 +169,52 @@ compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_sta
     if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
 }
 
+// In place, anchored at the END of every unit's region (position ranking only): the kept set is
+// the `head` leading rows plus the suffix [n - (b - head), n), so it is enough to lift the leading
+// rows to just below the suffix; the compacted cache of the unit is then rows [n - b, n) of its
+// own region.  At most `sink` rows move per unit.  The move is upwards and may overlap itself
+// (n - b < head), so the rows go in blocks of 256 pieces from the top down, each block loaded by
+// all threads before any of it is stored; a block's destinations lie above everything that the
+// blocks after it still have to read.
+__global__ void __launch_bounds__(kThreads)
+compact_inplace_back_kernel(refree_params p, char *k, char *v, const int32_t *seq_start, const int32_t *seq_len,
+                            const int64_t *offsets, int32_t *dev_status)
+{
+    const int Hkv = p.num_kv_heads;
+    const int u = blockIdx.x, s = u / Hkv, g = u % Hkv;
+    const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const int vec_per_row = (p.head_dim * esz) >> 4;
+    const int vshift = 31 - __clz(vec_per_row);
+    const int n = max(seq_len[s], 0);
+    const int64_t off = offsets[u], b64 = offsets[u + 1] - off;
+    if (off < 0 || b64 < 0 || b64 > n) {
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
+        return;
+    }
+    const int b = (int)b64, head = min(b, min(p.sink, n)), shift = n - b;
+    if (shift == 0 || head == 0) return;
+    const int64_t tok0 = seq_start[s];
+    char *kb = k + ((int64_t)s * p.k_stride_seq + tok0 * p.k_stride_tok + (int64_t)g * p.k_stride_head) * esz;
+    char *vb = v + ((int64_t)s * p.v_stride_seq + tok0 * p.v_stride_tok + (int64_t)g * p.v_stride_head) * esz;
+    const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
+    const int total_vec = head << vshift;
+    for (int c0 = (total_vec - 1) / kThreads * kThreads; c0 >= 0; c0 -= kThreads) {
+        const int e = c0 + threadIdx.x;
+        const bool on = e < total_vec;
+        const int row = e >> vshift, c = e & (vec_per_row - 1);
+        int4 kv = {}, vv = {};
+        if (on) {
+            kv = __ldcg(reinterpret_cast<const int4 *>(kb + (int64_t)row * k_tok + c * 16));
+            vv = __ldcg(reinterpret_cast<const int4 *>(vb + (int64_t)row * v_tok + c * 16));
+        }
+        __syncthreads();
+        if (on) {
+            *reinterpret_cast<int4 *>(kb + (int64_t)(row + shift) * k_tok + c * 16) = kv;
+            *reinterpret_cast<int4 *>(vb + (int64_t)(row + shift) * v_tok + c * 16) = vv;
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
@@ -200,8 +246,14 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
 
 cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, const int32_t *seq_start,
                                    const int32_t *seq_len, const int64_t *offsets, const int32_t *kept_idx,
-                                   bool position_ranges, int32_t *dev_status, cudaStream_t st)
+                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st)
 {
+    if (anchor_back) {
+        compact_inplace_back_kernel<<<p.num_seqs * p.num_kv_heads, kThreads, 0, st>>>(
+            p, (char *)k, (char *)v, seq_start, seq_len, offsets, dev_status);
+        count_launches(1);
+        return cudaGetLastError();
+    }
     static int grid_blocks[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);

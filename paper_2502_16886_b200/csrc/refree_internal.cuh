@@ -154,7 +154,7 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
 
 cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, const int32_t *seq_start,
                                    const int32_t *seq_len, const int64_t *offsets, const int32_t *kept_idx,
-                                   bool position_ranges, int32_t *dev_status, cudaStream_t st);
+                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st);
 
 size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,

@@ -2,10 +2,11 @@
 
 The oracle's selection (budgets, offsets, kept positions) and its dense compacted
 cache are computed on the CPU; the kernel is then given the oracle's selection and
-must leave, at the front of every unit's own region of K and V, exactly the rows
-the oracle compacted (bit compare).  Sizes span several rounds of the kernel (one
-round is what the whole grid holds in registers, about 38 K rows of 256 bytes)
-and ragged tails; both rankings, both layouts, both storage types.
+must leave, at the front (or, for position ranking, optionally at the end) of every
+unit's own region of K and V, exactly the rows the oracle compacted (bit compare).
+Sizes span several rounds of the front-anchored kernel (one round is what the whole
+grid holds in registers, about 38 K rows of 256 bytes) and ragged tails; both
+rankings, both layouts, both storage types.
 """
 import dataclasses
 
@@ -31,10 +32,12 @@ def _cfg(**kw):
     return dataclasses.replace(workloads.CONFIGS[0], **kw)
 
 
-def _unit_rows(t, lay, s, g, count):
-    """First ``count`` rows of unit (s, g)'s own region of a cache tensor laid out like ``lay``."""
+def _unit_rows(t, lay, s, g, count, back=False):
+    """First (or, ``back``, last) ``count`` rows of unit (s, g)'s own region of a cache tensor laid out like ``lay``."""
     view = t.permute(1, 0, 2) if lay.layout == "token_major" else t
     a = int(lay.seq_start[s])
+    if back:
+        a += int(lay.seq_len[s]) - count
     return view[g, a:a + count]
 
 
@@ -45,7 +48,7 @@ def _selection(p, lay, rng, power):
     return orc.select(parity.oracle_params(p), scores, lay.seq_len)
 
 
-def _run_inplace_and_check(p, lay, sel):
+def _run_inplace_and_check(p, lay, sel, anchor=binding.ANCHOR_FRONT):
     op = parity.oracle_params(p)
     want_k, want_v = orc.compact(op, lay.k, lay.v, lay.seq_start, lay.seq_len, sel)
     k, v = lay.k.to(DEV), lay.v.to(DEV)
@@ -54,18 +57,19 @@ def _run_inplace_and_check(p, lay, sel):
     kept = torch.from_numpy(sel.kept_idx if sel.kept_idx.size else np.zeros(1, np.int32)).to(DEV)
     ranges = p.rank_mode == binding.RANK_POSITION or p.force_full
     binding.refree_compact_inplace(p, k, v, lay.seq_start.to(DEV), lay.seq_len.to(DEV), offsets,
-                                   None if ranges else kept, status)
+                                   None if ranges else kept, status, anchor=anchor)
     torch.cuda.synchronize()
     assert status.item() == 0
     k, v = k.cpu(), v.cpu()
     moved = 0
+    back = anchor == binding.ANCHOR_BACK
     for s in range(p.num_seqs):
         for g in range(p.num_kv_heads):
             u = s * p.num_kv_heads + g
             a, b = int(sel.offsets[u]), int(sel.offsets[u + 1])
             assert b - a == int(sel.lengths[s, g])
-            assert torch.equal(parity.bits(_unit_rows(k, lay, s, g, b - a)), parity.bits(want_k[a:b]))
-            assert torch.equal(parity.bits(_unit_rows(v, lay, s, g, b - a)), parity.bits(want_v[a:b]))
+            assert torch.equal(parity.bits(_unit_rows(k, lay, s, g, b - a, back)), parity.bits(want_k[a:b]))
+            assert torch.equal(parity.bits(_unit_rows(v, lay, s, g, b - a, back)), parity.bits(want_v[a:b]))
             moved += b - a
     return moved
 
@@ -90,6 +94,38 @@ def test_inplace_compaction_small_budgets_and_short_sequences(rank_mode):
     lay = workloads.make_layer(cfg, 0, seq_lens=[3, 4, 5, 12, 13, 700, 2049])
     p = binding.params_for(cfg, lay, rank_mode=rank_mode, threshold=0.6)
     _run_inplace_and_check(p, lay, _selection(p, lay, np.random.default_rng(6), power=8))
+
+
+@pytest.mark.parametrize("layout,dtype,d", [("head_major", "bf16", 128), ("token_major", "bf16", 128),
+                                            ("head_major", "fp32", 64)])
+@pytest.mark.parametrize("sink,threshold", [(4, 0.02), (4, 0.6), (0, 0.1), (40, 0.3), (700, 0.05)])
+def test_inplace_anchored_at_the_end_lifts_only_the_leading_rows(layout, dtype, d, sink, threshold):
+    """Position ranking, compacted cache in rows [n - b, n): against the oracle's dense output.  Sink counts
+    from none to more rows than one block of the kernel moves at once, budgets that make the lifted rows
+    overlap their own sources (n - b < sink) and budgets that do not."""
+    cfg = _cfg(window=8, dtype=dtype, head_dim=d, num_q_heads=4, num_kv_heads=2, sink=sink)
+    lay = workloads.make_layer(cfg, 2, layout=layout, seq_lens=[5000, 3, 0, 41, 709, 1, 2300])
+    p = binding.params_for(cfg, lay, threshold=threshold)
+    sel = _selection(p, lay, np.random.default_rng(11), power=4)
+    shifts = [int(n) - int(b) for n, row in zip(lay.seq_len.tolist(), sel.lengths.tolist()) for b in row]
+    assert any(x > 0 for x in shifts)
+    if sink == 700:
+        assert any(0 < x < 700 for x in shifts)      # a self-overlapping move of several blocks
+    _run_inplace_and_check(p, lay, sel, anchor=binding.ANCHOR_BACK)
+
+
+def test_inplace_anchored_at_the_end_is_for_position_ranking_only():
+    cfg = _cfg(window=8, dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[100])
+    p = binding.params_for(cfg, lay, rank_mode=binding.RANK_SCORE)
+    k, v = lay.k.to(DEV), lay.v.to(DEV)
+    off = torch.tensor([0, 50], dtype=torch.int64, device=DEV)
+    kept = torch.arange(50, dtype=torch.int32, device=DEV)
+    rc = binding.refree_compact_inplace(p, k, v, lay.seq_start.to(DEV), lay.seq_len.to(DEV), off, kept, check=False,
+                                        anchor=binding.ANCHOR_BACK)
+    assert rc == binding.ERR_UNSUPPORTED
+    assert binding.refree_compact_inplace(p, k, v, lay.seq_start.to(DEV), lay.seq_len.to(DEV), off, kept, check=False,
+                                          anchor=7) == binding.ERR_INVALID_ARG
 
 
 def test_inplace_compaction_of_a_frozen_layer_changes_nothing():

@@ -398,6 +398,26 @@ def run_ours(args):
                 "bytes_per_layer": int(bytes_layer), "achieved": round(gbs, 1), "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(gbs / peak, 4)}
 
+    def fused_inplace_ms():
+        """The whole pass with end-anchored in-place compaction, one call per layer (overwrites the cache)."""
+        ln, of = layers[0]["lengths"], layers[0]["offsets"]
+
+        def call(d):
+            binding.refree_compress_layer_inplace(params, d["q"], d["k"], d["v"], seq_start, seq_len, total, ln, of,
+                                                  binding.ANCHOR_BACK, ws, status)
+        for d in layers:
+            call(d)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for d in layers:
+                call(d)
+        e1.record()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, f"device status {int(status.item())}"
+        return e0.elapsed_time(e1) / (reps * L)
+
     if rank_mode == binding.RANK_POSITION:
         lifted_rows = units * min(cfg.sink, min(seq_lens))
         inplace_line = [
@@ -405,6 +425,9 @@ def run_ours(args):
                              4 * lifted_rows * row),
             inplace_line_for(binding.ANCHOR_FRONT, "anchored at the front (every kept row moves)",
                              stage_bytes["compact"])]
+        fms = fused_inplace_ms()
+        inplace_line.append({"kernel": "refree_compress_layer_inplace, anchored at the end (whole pass per layer)",
+                             "ms_per_layer": round(fms, 5), "tokens_per_s_per_layer": round(total / (fms * 1e-3), 1)})
     else:
         inplace_line = None
 

@@ -174,6 +174,19 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
                                     void *workspace, size_t workspace_bytes,
                                     int32_t *device_status, void *stream);
 
+/* The whole per-layer pass with the compaction done in place: score -> select
+ * -> refree_compact_inplace, enqueued back to back on `stream`.  k and v are
+ * read by the scoring and then rewritten; lengths and offsets are outputs as in
+ * refree_compress_layer; `anchor` and the resulting layout are those of
+ * refree_compact_inplace (REFREE_ANCHOR_BACK needs position ranking or
+ * force_full).  With position ranking and REFREE_ANCHOR_BACK the pass costs
+ * little more than its scoring stage.  workspace as for refree_compress_layer. */
+refree_status refree_compress_layer_inplace(const refree_params *p, const void *q_win, void *k, void *v,
+                                            const int32_t *seq_start, const int32_t *seq_len,
+                                            int64_t total_tokens, int32_t *lengths, int64_t *offsets,
+                                            int32_t anchor, void *workspace, size_t workspace_bytes,
+                                            int32_t *device_status, void *stream);
+
 /* The pass of Algorithm 1 for a run of `num_layers` device-resident layers that
  * share one shape (Section 3.3: the cache of every layer is compressed once,
  * after prefill).  Scoring is bound by the tensor pipes and compaction by HBM,

@@ -89,6 +89,8 @@ SIGNATURES = {
     "refree_select_budget_static": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, _VP, _VP]),
+    "refree_compress_layer_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, ctypes.c_int32, _VP, _SZ,
+                                                     _VP, _VP]),
     "refree_compress_layer": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP,
                                              _VP, _VP, _VP, _SZ, _VP, _VP]),
     "refree_layers_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
@@ -212,6 +214,18 @@ def refree_compact_inplace(p: Params, k, v, seq_start, seq_len, offsets, kept_id
                                       _dp(kept_idx), anchor, _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_compact_inplace")
+    return rc
+
+
+def refree_compress_layer_inplace(p: Params, q_win, k, v, seq_start, seq_len, total_tokens, lengths, offsets, anchor,
+                                  workspace, device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_compress_layer_inplace(ctypes.byref(c), _dp(q_win), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len),
+                                             total_tokens, _dp(lengths), _dp(offsets), anchor, _dp(workspace),
+                                             workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                             _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compress_layer_inplace")
     return rc
 
 

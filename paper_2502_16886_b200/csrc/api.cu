@@ -316,6 +316,44 @@ refree_status refree_compress_layer(const refree_params *p, const void *q_win,
                          offsets, kept_idx, scores, (char *)workspace, lay, device_status, cs, cs, nullptr);
 }
 
+refree_status refree_compress_layer_inplace(const refree_params *p, const void *q_win, void *k, void *v,
+                                            const int32_t *seq_start, const int32_t *seq_len,
+                                            int64_t total_tokens, int32_t *lengths, int64_t *offsets,
+                                            int32_t anchor, void *workspace, size_t workspace_bytes,
+                                            int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, total_tokens);
+    if (st != REFREE_OK) return st;
+    if (!q_win || !k || !v || !seq_start || !seq_len || !lengths || !offsets) return REFREE_ERR_INVALID_ARG;
+    if (anchor != REFREE_ANCHOR_FRONT && anchor != REFREE_ANCHOR_BACK) return REFREE_ERR_INVALID_ARG;
+    const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
+    if (!ranges && anchor == REFREE_ANCHOR_BACK) return REFREE_ERR_UNSUPPORTED;
+    st = check_kv_layout(p, k, v, true);
+    if (st != REFREE_OK) return st;
+    const Workspace lay = workspace_layout(*p, total_tokens);
+    if (!workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    char *ws = (char *)workspace;
+    cudaStream_t cs = (cudaStream_t)stream;
+    float *sc = reinterpret_cast<float *>(ws + lay.scores_off);
+    int32_t *kept = ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off);
+    GroupPartial *groups = nullptr;
+    if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
+        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
+        groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
+    cudaError_t e = cudaSuccess;
+    if (total_tokens > 0 && !p->force_full)
+        e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    // the end-anchored kernel forms the offsets itself: no emit launch
+    const bool lean = anchor == REFREE_ANCHOR_BACK;
+    e = launch_select(*p, sc, seq_len, total_tokens, lengths, offsets, kept, (int64_t)p->num_kv_heads * total_tokens, ws,
+                      lay, device_status, cs, !lean, groups);
+    if (e != cudaSuccess) return REFREE_ERR_CUDA;
+    return from_cuda(launch_compact_inplace(*p, k, v, seq_start, seq_len, offsets, kept, ranges, lean, device_status, cs,
+                                            lean ? lengths : nullptr, lean ? offsets : nullptr));
+}
+
 // ---- a run of device-resident layers, compaction of layer l under the scoring of layer l + 1 ----
 namespace {
 struct LayerPipe {

@@ -178,15 +178,34 @@ compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_sta
 // blocks after it still have to read.
 __global__ void __launch_bounds__(kThreads)
 compact_inplace_back_kernel(refree_params p, char *k, char *v, const int32_t *seq_start, const int32_t *seq_len,
-                            const int64_t *offsets, int32_t *dev_status)
+                            const int64_t *offsets, const int32_t *lengths, int64_t *offsets_out, int32_t *dev_status)
 {
+    __shared__ long long s_part[kThreads / 32];
     const int Hkv = p.num_kv_heads;
     const int u = blockIdx.x, s = u / Hkv, g = u % Hkv;
     const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
     const int vec_per_row = (p.head_dim * esz) >> 4;
     const int vshift = 31 - __clz(vec_per_row);
     const int n = max(seq_len[s], 0);
-    const int64_t off = offsets[u], b64 = offsets[u + 1] - off;
+    int64_t off, b64;
+    if (lengths) {
+        // fused pass: budgets come straight from the selection, and the running sum is formed here
+        long long part = 0;
+        for (int t = threadIdx.x; t < u; t += kThreads) part += lengths[t];
+        for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = part;
+        __syncthreads();
+        off = 0;
+        for (int wv = 0; wv < kThreads / 32; ++wv) off += s_part[wv];
+        b64 = lengths[u];
+        if (threadIdx.x == 0) {
+            offsets_out[u] = off;
+            if (u == (int)gridDim.x - 1) offsets_out[u + 1] = off + b64;
+        }
+    } else {
+        off = offsets[u];
+        b64 = offsets[u + 1] - off;
+    }
     if (off < 0 || b64 < 0 || b64 > n) {
         if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
         return;
@@ -246,11 +265,12 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
 
 cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, const int32_t *seq_start,
                                    const int32_t *seq_len, const int64_t *offsets, const int32_t *kept_idx,
-                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st)
+                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st,
+                                   const int32_t *lengths, int64_t *offsets_out)
 {
     if (anchor_back) {
         compact_inplace_back_kernel<<<p.num_seqs * p.num_kv_heads, kThreads, 0, st>>>(
-            p, (char *)k, (char *)v, seq_start, seq_len, offsets, dev_status);
+            p, (char *)k, (char *)v, seq_start, seq_len, offsets, lengths, offsets_out, dev_status);
         count_launches(1);
         return cudaGetLastError();
     }

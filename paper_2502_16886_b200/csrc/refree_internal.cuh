@@ -152,9 +152,12 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
                            int64_t capacity_rows, int32_t *dev_status, cudaStream_t st,
                            bool beside_scoring = false);
 
+// With `lengths` and `offsets_out` (end-anchored form only) the kernel takes the budgets from `lengths` and
+// writes their running sum itself, so the selection need not emit offsets first.
 cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, const int32_t *seq_start,
                                    const int32_t *seq_len, const int64_t *offsets, const int32_t *kept_idx,
-                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st);
+                                   bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st,
+                                   const int32_t *lengths = nullptr, int64_t *offsets_out = nullptr);
 
 size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,

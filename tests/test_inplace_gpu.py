@@ -165,6 +165,38 @@ def test_inplace_after_the_library_selection_equals_the_out_of_place_pass():
                                    parity.bits(res.v_out[off[u]:off[u + 1]].cpu()))
 
 
+@pytest.mark.parametrize("rank_mode,anchor,window,dtype", [
+    (binding.RANK_POSITION, binding.ANCHOR_BACK, 16, "bf16"), (binding.RANK_POSITION, binding.ANCHOR_FRONT, 16, "bf16"),
+    (binding.RANK_SCORE, binding.ANCHOR_FRONT, 16, "bf16"), (binding.RANK_POSITION, binding.ANCHOR_BACK, 1, "bf16"),
+    (binding.RANK_POSITION, binding.ANCHOR_BACK, 8, "fp32")])
+def test_fused_inplace_pass_against_the_oracle(rank_mode, anchor, window, dtype):
+    """refree_compress_layer_inplace: budgets equal to the oracle's and, in every unit's own region, the rows
+    of the oracle's dense compacted cache (tensor-core, single-row and generic scoring paths)."""
+    cfg = _cfg(window=window, dtype=dtype, head_dim=128, num_q_heads=8, num_kv_heads=2)
+    lay = workloads.make_layer(cfg, 4, seq_lens=[3000, 130, 0, 777])
+    p = binding.params_for(cfg, lay, rank_mode=rank_mode, threshold=0.05)
+    ref = orc.compress_layer(parity.oracle_params(p), lay.q_win, lay.k, lay.v, lay.seq_start, lay.seq_len)
+    q, k, v, ss, sl = [t.to(DEV) for t in (lay.q_win, lay.k, lay.v, lay.seq_start, lay.seq_len)]
+    units = p.num_seqs * p.num_kv_heads
+    lengths = torch.zeros(units, dtype=torch.int32, device=DEV)
+    offsets = torch.zeros(units + 1, dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.empty(binding.refree_workspace_size(p, lay.total_tokens), dtype=torch.uint8, device=DEV)
+    binding.refree_compress_layer_inplace(p, q, k, v, ss, sl, lay.total_tokens, lengths, offsets, anchor, ws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert lengths.cpu().tolist() == ref.sel.lengths.reshape(-1).tolist()
+    assert offsets.cpu().tolist() == ref.sel.offsets.tolist()
+    kc, vc = k.cpu(), v.cpu()
+    back = anchor == binding.ANCHOR_BACK
+    for s in range(p.num_seqs):
+        for g in range(p.num_kv_heads):
+            u = s * p.num_kv_heads + g
+            a, b = int(ref.sel.offsets[u]), int(ref.sel.offsets[u + 1])
+            assert torch.equal(parity.bits(_unit_rows(kc, lay, s, g, b - a, back)), parity.bits(ref.k_out[a:b]))
+            assert torch.equal(parity.bits(_unit_rows(vc, lay, s, g, b - a, back)), parity.bits(ref.v_out[a:b]))
+
+
 def test_inplace_flags_offsets_that_do_not_fit_the_sequences():
     cfg = _cfg(window=8, dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1)
     lay = workloads.make_layer(cfg, 0, seq_lens=[100])

@@ -124,6 +124,31 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
                              const int32_t *kept_idx, void *k_out, void *v_out,
                              int64_t capacity_rows, int32_t *device_status, void *stream);
 
+/* Step S7 into a paged cache (Section 3.3 batches sequences whose budgets
+ * differ; a paged serving cache holds such ragged lengths in fixed-size blocks).
+ * Row t of unit u = s*num_kv_heads + g, i.e. the row refree_compact would write
+ * to k_out[offsets[u] + t], goes to
+ *     k_pool[block_table[u * max_blocks_per_unit + t / block_rows], t % block_rows, :]
+ * and the same for V; rows are copied bit for bit.
+ *   lengths      [num_seqs*num_kv_heads] int32 budgets (device, in)
+ *   offsets, kept_idx  as produced by refree_select_budget; both ignored (may be
+ *                null) with position ranking or force_full, required with score ranking
+ *   block_table  [num_seqs*num_kv_heads, max_blocks_per_unit] int32 block numbers
+ *                (device, in); the caller assigns ceil(n / block_rows) blocks per
+ *                unit before the call (the budgets are only known on the device)
+ *                and can release those beyond ceil(lengths[u] / block_rows) later
+ *   k_pool, v_pool  [num_blocks, block_rows, head_dim], params->dtype, 16-byte
+ *                aligned (device, out); must not overlap K or V
+ * A budget above max_blocks_per_unit * block_rows or the sequence length, or a
+ * block number outside [0, num_blocks), sets REFREE_DEV_CAPACITY in
+ * *device_status; the rows concerned are not written. */
+refree_status refree_compact_paged(const refree_params *p, const void *k, const void *v,
+                                   const int32_t *seq_start, const int32_t *seq_len,
+                                   const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
+                                   const int32_t *block_table, int32_t max_blocks_per_unit, int32_t block_rows,
+                                   void *k_pool, void *v_pool, int64_t num_blocks,
+                                   int32_t *device_status, void *stream);
+
 /* Step S7 in place, for callers with no room for a second copy of the cache.
  * The kept rows of every unit end up contiguous inside the unit's OWN region of
  * K and V (same strides as the input), bit for bit the rows refree_compact would

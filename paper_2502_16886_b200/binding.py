@@ -88,6 +88,8 @@ SIGNATURES = {
     "refree_select_budget": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _SZ, _VP, _VP]),
     "refree_select_budget_static": (ctypes.c_int, [_PP, _VP, _VP, _I64, _VP, _VP, _VP, _I64, _VP, _VP]),
     "refree_compact": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP]),
+    "refree_compact_paged": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, ctypes.c_int32,
+                                            _VP, _VP, _I64, _VP, _VP]),
     "refree_compact_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, _VP, _VP]),
     "refree_compress_layer_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, ctypes.c_int32, _VP, _SZ,
                                                      _VP, _VP]),
@@ -203,6 +205,18 @@ def refree_compact(p: Params, k, v, seq_start, seq_len, lengths, offsets, kept_i
                               _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_compact")
+    return rc
+
+
+def refree_compact_paged(p: Params, k, v, seq_start, seq_len, lengths, offsets, kept_idx, block_table, block_rows,
+                         k_pool, v_pool, device_status=None, stream=None, check=True) -> int:
+    """``block_table`` is int32 ``[units, max_blocks_per_unit]``; the pools are ``[num_blocks, block_rows, d]``."""
+    c = p.c_struct()
+    rc = lib().refree_compact_paged(ctypes.byref(c), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len), _dp(lengths),
+                                    _dp(offsets), _dp(kept_idx), _dp(block_table), block_table.shape[1], block_rows,
+                                    _dp(k_pool), _dp(v_pool), k_pool.shape[0], _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_compact_paged")
     return rc
 
 

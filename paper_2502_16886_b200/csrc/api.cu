@@ -194,6 +194,29 @@ refree_status refree_compact(const refree_params *p, const void *k, const void *
                                     v_out, capacity_rows, device_status, (cudaStream_t)stream));
 }
 
+refree_status refree_compact_paged(const refree_params *p, const void *k, const void *v,
+                                   const int32_t *seq_start, const int32_t *seq_len,
+                                   const int32_t *lengths, const int64_t *offsets, const int32_t *kept_idx,
+                                   const int32_t *block_table, int32_t max_blocks_per_unit, int32_t block_rows,
+                                   void *k_pool, void *v_pool, int64_t num_blocks,
+                                   int32_t *device_status, void *stream)
+{
+    refree_status st = check_params(p, 0);
+    if (st != REFREE_OK) return st;
+    if (!k || !v || !seq_start || !seq_len || !lengths || !block_table || !k_pool || !v_pool ||
+        max_blocks_per_unit < 1 || block_rows < 1 || num_blocks < 0)
+        return REFREE_ERR_INVALID_ARG;
+    const bool ranges = p->rank_mode == REFREE_RANK_POSITION || p->force_full;
+    if (!ranges && (!kept_idx || !offsets)) return REFREE_ERR_INVALID_ARG;
+    st = check_kv_layout(p, k, v, true);
+    if (st != REFREE_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(k_pool) & 15) || (reinterpret_cast<uintptr_t>(v_pool) & 15))
+        return REFREE_ERR_UNSUPPORTED;
+    return from_cuda(launch_compact_paged(*p, k, v, seq_start, seq_len, lengths, offsets, ranges ? nullptr : kept_idx,
+                                          ranges, block_table, max_blocks_per_unit, block_rows, k_pool, v_pool,
+                                          num_blocks, device_status, (cudaStream_t)stream));
+}
+
 refree_status refree_compact_inplace(const refree_params *p, void *k, void *v,
                                      const int32_t *seq_start, const int32_t *seq_len,
                                      const int64_t *offsets, const int32_t *kept_idx, int32_t anchor,

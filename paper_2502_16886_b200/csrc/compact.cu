@@ -234,6 +234,66 @@ compact_inplace_back_kernel(refree_params p, char *k, char *v, const int32_t *se
     }
 }
 
+// Paged form of the same step: row t of unit u goes to row t % block_rows of the block
+// block_table[u][t / block_rows] of a pool of fixed-size blocks (the layout of a paged
+// serving cache).  Same gather as compact_kernel; only the destination address differs.
+__global__ void __launch_bounds__(kThreads)
+compact_paged_kernel(refree_params p, const char *k, const char *v, const int32_t *seq_start,
+                     const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
+                     const int32_t *kept_idx, int position_ranges, const int32_t *block_table,
+                     int max_blocks_per_unit, int block_rows, char *k_pool, char *v_pool, int64_t num_blocks,
+                     int32_t *dev_status)
+{
+    const int Hkv = p.num_kv_heads;
+    const int u = blockIdx.y, s = u / Hkv, g = u % Hkv;
+    const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+    const int row_bytes = p.head_dim * esz;
+    const int vec_per_row = row_bytes >> 4;
+    const int vshift = 31 - __clz(vec_per_row);
+    const int n = max(seq_len[s], 0);
+    const int b = lengths[u];
+    if (b < 0 || b > n || (int64_t)b > (int64_t)max_blocks_per_unit * block_rows || (kept_idx && offsets[u] < 0)) {
+        if (threadIdx.x == 0 && blockIdx.x == 0 && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
+        return;
+    }
+    const int head = min(b, min(p.sink, n));
+    const int64_t tok0 = seq_start[s];
+    const char *kb = k + ((int64_t)s * p.k_stride_seq + tok0 * p.k_stride_tok + (int64_t)g * p.k_stride_head) * esz;
+    const char *vb = v + ((int64_t)s * p.v_stride_seq + tok0 * p.v_stride_tok + (int64_t)g * p.v_stride_head) * esz;
+    const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
+    const int32_t *idx = kept_idx ? kept_idx + offsets[u] : nullptr;
+    const int32_t *table = block_table + (int64_t)u * max_blocks_per_unit;
+    const int64_t nvec = (int64_t)b << vshift;
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    bool bad = false;
+    for (int64_t e0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; e0 < nvec; e0 += stride * kUnroll) {
+        int4 kv[kUnroll], vv[kUnroll];
+        int64_t dst[kUnroll];
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r) {
+            const int64_t e = e0 + r * stride;
+            dst[r] = -1;
+            if (e < nvec) {
+                const int t = (int)(e >> vshift), c = (int)(e & (vec_per_row - 1));
+                const int src = position_ranges ? (t < head ? t : n - b + t) : idx[t];
+                const int blk = __ldg(table + t / block_rows);
+                if (blk < 0 || blk >= num_blocks || src < 0 || src >= n) { bad = true; continue; }
+                kv[r] = *reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok + c * 16);
+                vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16));
+                dst[r] = ((int64_t)blk * block_rows + t % block_rows) * row_bytes + c * 16;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r) {
+            if (dst[r] >= 0) {
+                st_stream(reinterpret_cast<int4 *>(k_pool + dst[r]), kv[r]);
+                st_stream(reinterpret_cast<int4 *>(v_pool + dst[r]), vv[r]);
+            }
+        }
+    }
+    if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_CAPACITY);
+}
+
 }  // namespace
 
 cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
@@ -296,6 +356,22 @@ cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, con
     void *args[9] = {&pv, &kc, &vc, &seq_start, &seq_len, &offsets, &kept_idx, &ranges, &dev_status};
     e = cudaLaunchCooperativeKernel((const void *)compact_inplace_kernel, dim3(grid_blocks[dev]), dim3(kThreads), args, 0, st);
     if (e != cudaSuccess) return e;
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compact_paged(const refree_params &p, const void *k, const void *v, const int32_t *seq_start,
+                                 const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
+                                 const int32_t *kept_idx, bool position_ranges, const int32_t *block_table,
+                                 int max_blocks_per_unit, int block_rows, void *k_pool, void *v_pool,
+                                 int64_t num_blocks, int32_t *dev_status, cudaStream_t st)
+{
+    const int U = p.num_seqs * p.num_kv_heads;
+    const int gx = max(1, (148 * 8) / U);
+    compact_paged_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
+                                                           lengths, offsets, kept_idx, position_ranges ? 1 : 0,
+                                                           block_table, max_blocks_per_unit, block_rows,
+                                                           (char *)k_pool, (char *)v_pool, num_blocks, dev_status);
     count_launches(1);
     return cudaGetLastError();
 }

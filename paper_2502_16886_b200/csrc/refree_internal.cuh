@@ -159,6 +159,12 @@ cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, con
                                    bool position_ranges, bool anchor_back, int32_t *dev_status, cudaStream_t st,
                                    const int32_t *lengths = nullptr, int64_t *offsets_out = nullptr);
 
+cudaError_t launch_compact_paged(const refree_params &p, const void *k, const void *v, const int32_t *seq_start,
+                                 const int32_t *seq_len, const int32_t *lengths, const int64_t *offsets,
+                                 const int32_t *kept_idx, bool position_ranges, const int32_t *block_table,
+                                 int max_blocks_per_unit, int block_rows, void *k_pool, void *v_pool,
+                                 int64_t num_blocks, int32_t *dev_status, cudaStream_t st);
+
 size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,
                                     const int64_t *offsets, int64_t max_rows, float *out, void *workspace,

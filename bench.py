@@ -338,6 +338,27 @@ def run_ours(args):
                 "ms_per_launch": round(stage_ms[dominant], 5),
                 "stages_ms": {k: round(v, 5) for k, v in stage_ms.items()},
                 "stages_gbs": {k: round(stage_bytes[k] / (stage_ms[k] * 1e-3) / 1e9, 1) for k in stage_ms}}
+    if dominant == "score" and cfg.window > 1 and cfg.dtype == "bf16":
+        # the scoring stage's three roofs (it forms the logits twice): K once from HBM, the dense contraction
+        # at the measured bf16 GEMM rate, one exponential per logit at 16 per clock per SM
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except Exception:
+            pass
+        tf_peak = float(peaks.get("bf16_tflops", 1590.0))
+        sm_hz = float(peaks.get("sm_max_mhz", 1965.0)) * 1e6
+        logits = 2.0 * cfg.num_kv_heads * total * cfg.group * cfg.window          # both passes
+        t_hbm = stage_bytes["score"] / (peak * 1e9) * 1e6
+        t_mma = logits * 2 * cfg.head_dim / (tf_peak * 1e12) * 1e6
+        t_exp = logits / (148 * 16 * sm_hz) * 1e6
+        bound_us = max(t_hbm, t_mma, t_exp)
+        roofline["other_roofs"] = {
+            "us": {"hbm": round(t_hbm, 2), "tensor": round(t_mma, 2), "exp": round(t_exp, 2)},
+            "binding": max((("hbm", t_hbm), ("tensor", t_mma), ("exp", t_exp)), key=lambda kv: kv[1])[0],
+            "frac_of_binding": round(bound_us / (stage_ms["score"] * 1e3), 4),
+            "tensor_tflops": round(logits * 2 * cfg.head_dim / (stage_ms["score"] * 1e-3) / 1e12, 1),
+            "tensor_peak_tflops": tf_peak}
     roofline_pass = {"bound": "hbm", "achieved": round(pass_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}",
                      "unit": "GB/s", "frac": round(pass_gbs / peak, 4), "frac_of_8TBps": round(pass_gbs / 8000.0, 4),
                      "bytes_per_layer": int(bytes3), "bytes_per_layer_with_kept_k_reread": int(bytes4),

@@ -107,8 +107,9 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
 // reads only rows at or beyond its own destinations, which lie beyond every destination of
 // the rounds before it, so one grid barrier per round is all the ordering needed.
 constexpr int kUnrollInplace = 4;
+constexpr int kInplaceTable = 1024;   // running sums held in shared memory (8 KB)
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_start, const int32_t *seq_len,
                        const int64_t *offsets, const int32_t *kept_idx, int position_ranges, int32_t *dev_status)
 {
@@ -118,7 +119,15 @@ compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_sta
     const int esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
     const int vec_per_row = (p.head_dim * esz) >> 4;
     const int vshift = 31 - __clz(vec_per_row);
-    const int64_t total_vec = max((long long)__ldg(offsets + U), 0ll) << vshift;
+    // the running sums are searched once per piece: keep them in shared memory when they fit
+    __shared__ int64_t s_off[kInplaceTable];
+    const int64_t *tab = offsets;
+    if (U + 1 <= kInplaceTable) {
+        for (int i = threadIdx.x; i <= U; i += kThreads) s_off[i] = __ldg(offsets + i);
+        __syncthreads();
+        tab = s_off;
+    }
+    const int64_t total_vec = max((long long)tab[U], 0ll) << vshift;
     const int64_t lanes = (int64_t)gridDim.x * kThreads;
     const int64_t per_round = lanes * kUnrollInplace;
     const int64_t k_tok = p.k_stride_tok * esz, v_tok = p.v_stride_tok * esz;
@@ -136,12 +145,12 @@ compact_inplace_kernel(refree_params p, char *k, char *v, const int32_t *seq_sta
             int lo = 0, hi = U;                                       // unit whose rows contain `row`
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
-                if (__ldg(offsets + mid) <= row) lo = mid; else hi = mid;
+                if (tab[mid] <= row) lo = mid; else hi = mid;
             }
             const int u = lo, s = u / Hkv, g = u % Hkv;
-            const int64_t off = __ldg(offsets + u);
+            const int64_t off = tab[u];
             const int n = max(__ldg(seq_len + s), 0);
-            const int64_t b64 = __ldg(offsets + u + 1) - off;
+            const int64_t b64 = tab[u + 1] - off;
             const int t = (int)(row - off);
             if (off < 0 || b64 < 0 || b64 > n) { bad = true; continue; }
             const int b = (int)b64;

@@ -65,3 +65,50 @@ def test_decode_attention_over_the_compacted_layer_at_full_size(name):
     want = orc.decode_attention(op, q_new, res.k_out[:rows].cpu(), res.v_out[:rows].cpu(), res.offsets.cpu().numpy())
     np.testing.assert_allclose(out.cpu().numpy(), want, rtol=1e-4, atol=1e-4)
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name,n_layers", [("mistral7b_32k", 4), ("qwen25_7b_ragged8", 3)])
+def test_one_call_run_of_layers_at_full_size(name, n_layers):
+    """The step the benchmark times: refree_compress_layers over consecutive full-size layers (both
+    workspace halves reused).  Budgets and every compacted row against the oracle; a layer whose budgets
+    differ from the oracle's (near-ties, judged by the per-layer test above) is compared with the
+    per-layer call instead, which must agree with the one-call run bit for bit in any case."""
+    from oracle import refree_oracle as orc
+    cfg = workloads.get_config(name)
+    dev = "cuda:0"
+    lays = [workloads.make_layer(cfg, l) for l in range(n_layers)]
+    p = binding.params_for(cfg, lays[0])
+    total = lays[0].total_tokens
+    cap = p.num_kv_heads * total
+    units = p.num_seqs * p.num_kv_heads
+    q = [l.q_win.to(dev) for l in lays]
+    k = [l.k.to(dev) for l in lays]
+    v = [l.v.to(dev) for l in lays]
+    k_out = [torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype, device=dev) for _ in lays]
+    v_out = [torch.zeros(cap, p.head_dim, dtype=lays[0].k.dtype, device=dev) for _ in lays]
+    lengths = [torch.zeros(units, dtype=torch.int32, device=dev) for _ in lays]
+    offsets = [torch.zeros(units + 1, dtype=torch.int64, device=dev) for _ in lays]
+    ss, sl = lays[0].seq_start.to(dev), lays[0].seq_len.to(dev)
+    ws = torch.empty(binding.refree_layers_workspace_size(p, total), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.refree_compress_layers(p, binding.LayerPointers(q, k, v, k_out, v_out, lengths, offsets), ss, sl, total, cap,
+                                   ws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    exact = 0
+    for l, lay in enumerate(lays):
+        one = binding.compress_layer(p, q[l], k[l], v[l], ss, sl, total, want_scores=False, want_kept_idx=False)
+        torch.cuda.synchronize()
+        rows = int(offsets[l][-1])
+        assert torch.equal(lengths[l], one.lengths.reshape(-1)) and torch.equal(offsets[l], one.offsets)
+        assert torch.equal(parity.bits(k_out[l][:rows]), parity.bits(one.k_out[:rows]))
+        assert torch.equal(parity.bits(v_out[l][:rows]), parity.bits(one.v_out[:rows]))
+        ref = orc.compress_layer(parity.oracle_params(p), lay.q_win, lay.k, lay.v, lay.seq_start, lay.seq_len)
+        if np.array_equal(lengths[l].cpu().numpy(), ref.sel.lengths.reshape(-1)):
+            exact += 1
+            assert rows == int(ref.sel.offsets[-1])
+            assert torch.equal(parity.bits(k_out[l][:rows].cpu()), parity.bits(ref.k_out))
+            assert torch.equal(parity.bits(v_out[l][:rows].cpu()), parity.bits(ref.v_out))
+        del one
+    assert exact >= n_layers - 1, f"only {exact} of {n_layers} layers had the oracle's budgets exactly"
+    torch.cuda.empty_cache()

@@ -69,6 +69,48 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert rc == 2          # K not 16-byte aligned
 
 
+def test_host_side_validation_of_the_layer_run_inplace_and_paged_entry_points(lib):
+    good = binding.Params(1, 4, 2, 64, window=8, kv_tokens=128, k_strides=(0, 64, 8192), v_strides=(0, 64, 8192))
+    assert binding.refree_layers_workspace_size(good, 128) == 2 * binding.refree_workspace_size(good, 128)
+    c = good.c_struct()
+    fake = ctypes.c_void_p(4096)
+    one = (ctypes.c_void_p * 1)(4096)
+    null1 = (ctypes.c_void_p * 1)(None)
+    big = 1 << 30
+    # a run of layers: missing arrays, a null layer pointer, one workspace instead of two, nothing to do
+    assert lib.refree_compress_layers(ctypes.byref(c), 1, None, one, one, fake, fake, 128, one, one, 256, one, one,
+                                      fake, big, None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compress_layers(ctypes.byref(c), 1, one, null1, one, fake, fake, 128, one, one, 256, one, one,
+                                      fake, big, None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compress_layers(ctypes.byref(c), 1, one, one, one, fake, fake, 128, one, one, 256, one, one,
+                                      fake, binding.refree_workspace_size(good, 128), None, None) == binding.ERR_WORKSPACE
+    assert lib.refree_compress_layers(ctypes.byref(c), -1, one, one, one, fake, fake, 128, one, one, 256, one, one,
+                                      fake, big, None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compress_layers(ctypes.byref(c), 0, one, one, one, fake, fake, 128, one, one, 256, one, one,
+                                      fake, big, None, None) == binding.REFREE_OK
+    # in place: unknown anchor, end anchor with score ranking, score ranking without an index list
+    assert lib.refree_compact_inplace(ctypes.byref(c), fake, fake, fake, fake, fake, None, 2, None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compact_inplace(ctypes.byref(c), fake, None, fake, fake, fake, None, 0, None, None) == binding.ERR_INVALID_ARG
+    sc = binding.Params(**{**good.__dict__, "rank_mode": binding.RANK_SCORE}).c_struct()
+    assert lib.refree_compact_inplace(ctypes.byref(sc), fake, fake, fake, fake, fake, fake, binding.ANCHOR_BACK, None,
+                                      None) == binding.ERR_UNSUPPORTED
+    assert lib.refree_compact_inplace(ctypes.byref(sc), fake, fake, fake, fake, fake, None, binding.ANCHOR_FRONT, None,
+                                      None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compress_layer_inplace(ctypes.byref(sc), fake, fake, fake, fake, fake, 128, fake, fake,
+                                             binding.ANCHOR_BACK, fake, big, None, None) == binding.ERR_UNSUPPORTED
+    assert lib.refree_compress_layer_inplace(ctypes.byref(c), fake, fake, fake, fake, fake, 128, fake, fake,
+                                             binding.ANCHOR_BACK, None, 0, None, None) == binding.ERR_WORKSPACE
+    # paged: block geometry, missing table, unaligned pool, score ranking without offsets
+    assert lib.refree_compact_paged(ctypes.byref(c), fake, fake, fake, fake, fake, None, None, fake, 4, 0, fake, fake, 8,
+                                    None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compact_paged(ctypes.byref(c), fake, fake, fake, fake, fake, None, None, None, 4, 16, fake, fake, 8,
+                                    None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_compact_paged(ctypes.byref(c), fake, fake, fake, fake, fake, None, None, fake, 4, 16,
+                                    ctypes.c_void_p(4100), fake, 8, None, None) == binding.ERR_UNSUPPORTED
+    assert lib.refree_compact_paged(ctypes.byref(sc), fake, fake, fake, fake, fake, None, fake, fake, 4, 16, fake, fake, 8,
+                                    None, None) == binding.ERR_INVALID_ARG
+
+
 def test_missing_library_is_an_error(monkeypatch, lib):
     monkeypatch.setattr(binding, "_LIB", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/librefreekv.so")

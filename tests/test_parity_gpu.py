@@ -263,7 +263,7 @@ def test_pipelined_device_run_of_layers_matches_the_per_layer_call(rank_mode, wi
     caller's stream."""
     cfg = small_cfg(window=window, dtype=dtype, head_dim=128, num_q_heads=8, num_kv_heads=2)
     n_layers = 5
-    lays = [workloads.make_layer(cfg, l, seq_lens=[2700, 90, 1333]) for l in range(n_layers)]
+    lays = [workloads.make_layer(cfg, l, seq_lens=[2700, 0, 90, 1333, 1]) for l in range(n_layers)]
     p = binding.params_for(cfg, lays[0], rank_mode=rank_mode, threshold=0.05)
     total = lays[0].total_tokens
     cap = p.num_kv_heads * total

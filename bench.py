@@ -177,10 +177,10 @@ def algorithmic_bytes(cfg, seq_lens, lengths):
     return a, b4
 
 
-# dram__bytes_read + dram__bytes_write of one launch of the scoring kernel (ncu capture of the 8K workload,
-# summary under profiles/); traffic grows in proportion to the tokens, so the 32K figure is 4x the captured one.
-# Only for the kernel version the capture was taken on: window 64, tensor-core path.
-NCU_SCORE_TRAFFIC = {"llama3_8b_8k": 17_484_288, "mistral7b_32k": 4 * 17_484_288}
+# dram__bytes_read + dram__bytes_write of one launch of the scoring kernel, from the ncu captures summarised
+# under profiles/: the 32K layer captured at full size; the 8K layer captured on the 8-layer cut of its workload.
+# Only for the kernel version the captures were taken on: window 64, tensor-core path.
+NCU_SCORE_TRAFFIC = {"llama3_8b_8k": 17_484_288, "mistral7b_32k": 68_277_504 + 2_643_200}
 
 
 def ncu_traffic(cfg, stage):

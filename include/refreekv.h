@@ -344,6 +344,24 @@ refree_status refree_decode_attention(const refree_params *params, const void *q
                                       void *workspace, size_t workspace_bytes,
                                       int32_t *device_status, void *stream);
 
+/* The same decode step over the strided ragged cache that refree_compact_inplace
+ * (or refree_compress_layer_inplace) leaves: the rows of unit u = (s, g) are
+ * rows [0, lengths[u]) (REFREE_ANCHOR_FRONT) or [n_s - lengths[u], n_s)
+ * (REFREE_ANCHOR_BACK) of the unit's own region of k and v, addressed with
+ * seq_start and the strides of params as in refree_score.
+ *   k, v     the compacted-in-place cache arrays (device, in); head-major
+ *            layouts only: k_stride_tok = v_stride_tok = head_dim and the other
+ *            strides multiples of head_dim, else REFREE_ERR_UNSUPPORTED
+ *   lengths  [num_seqs*num_kv_heads] int32 budgets (device, in)
+ * Everything else as in refree_decode_attention. */
+refree_status refree_decode_attention_inplace(const refree_params *params, const void *q_new,
+                                              const void *k, const void *v,
+                                              const int32_t *seq_start, const int32_t *seq_len,
+                                              const int32_t *lengths, int32_t anchor,
+                                              int64_t max_rows_per_unit, float *out,
+                                              void *workspace, size_t workspace_bytes,
+                                              int32_t *device_status, void *stream);
+
 /* Diagnostic with no counterpart in the paper: the number of CUDA kernels this
  * library has enqueued in this process so far (all entry points, all streams). */
 int64_t refree_kernel_launch_count(void);

@@ -103,6 +103,8 @@ SIGNATURES = {
                                                    _I64, _VP, _VP, _VP, _SZ]),
     "refree_decode_workspace_size": (ctypes.c_int, [_PP, _I64, ctypes.POINTER(_SZ)]),
     "refree_decode_attention": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
+    "refree_decode_attention_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, _I64, _VP, _VP,
+                                                       _SZ, _VP, _VP]),
     "refree_host_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
     "refree_compress_layer_host": (ctypes.c_int, [_PP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP, _I64,
                                                   _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
@@ -274,6 +276,18 @@ def refree_decode_attention(p: Params, q_new, k_c, v_c, offsets, max_rows_per_un
                                        _dp(device_status), _stream(stream))
     if check:
         _check(rc, "refree_decode_attention")
+    return rc
+
+
+def refree_decode_attention_inplace(p: Params, q_new, k, v, seq_start, seq_len, lengths, anchor, max_rows_per_unit, out,
+                                    workspace, device_status=None, stream=None, check=True) -> int:
+    c = p.c_struct()
+    rc = lib().refree_decode_attention_inplace(ctypes.byref(c), _dp(q_new), _dp(k), _dp(v), _dp(seq_start), _dp(seq_len),
+                                               _dp(lengths), anchor, max_rows_per_unit, _dp(out), _dp(workspace),
+                                               workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                               _dp(device_status), _stream(stream))
+    if check:
+        _check(rc, "refree_decode_attention_inplace")
     return rc
 
 

@@ -274,6 +274,33 @@ refree_status refree_decode_attention(const refree_params *p, const void *q_new,
                                              device_status, (cudaStream_t)stream));
 }
 
+refree_status refree_decode_attention_inplace(const refree_params *p, const void *q_new,
+                                              const void *k, const void *v,
+                                              const int32_t *seq_start, const int32_t *seq_len,
+                                              const int32_t *lengths, int32_t anchor,
+                                              int64_t max_rows_per_unit, float *out,
+                                              void *workspace, size_t workspace_bytes,
+                                              int32_t *device_status, void *stream)
+{
+    refree_status st = check_decode(p, max_rows_per_unit);
+    if (st != REFREE_OK) return st;
+    if (!q_new || !k || !v || !seq_start || !seq_len || !lengths || !out) return REFREE_ERR_INVALID_ARG;
+    if (anchor != REFREE_ANCHOR_FRONT && anchor != REFREE_ANCHOR_BACK) return REFREE_ERR_INVALID_ARG;
+    st = check_kv_layout(p, k, v, true);
+    if (st != REFREE_OK) return st;
+    // the rows of a unit must be back to back, and every unit must start on a whole row
+    const int64_t d = p->head_dim;
+    if (p->k_stride_tok != d || p->v_stride_tok != d || p->k_stride_seq % d || p->k_stride_head % d ||
+        p->v_stride_seq % d || p->v_stride_head % d)
+        return REFREE_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < decode_workspace_bytes(*p, max_rows_per_unit) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return REFREE_ERR_WORKSPACE;
+    return from_cuda(launch_decode_attention(*p, q_new, k, v, nullptr, max_rows_per_unit, out, workspace, device_status,
+                                             (cudaStream_t)stream, seq_start, seq_len, lengths,
+                                             anchor == REFREE_ANCHOR_BACK));
+}
+
 // The launch sequence of one layer.  `cs` takes scoring and selection; compaction goes to `cc`
 // (after `scored`, recorded on `cs`, when the two differ).
 static refree_status enqueue_layer(const refree_params *p, const void *q_win, const void *k, const void *v,

@@ -41,6 +41,10 @@ struct DecArgs {
     refree_params p;
     const void *q, *kc, *vc;
     const int64_t *offsets;
+    // strided ragged cache (what refree_compact_inplace leaves): rows of unit (s, g) sit in the unit's own
+    // region of the original K / V arrays; `lengths` non-null selects this form and `offsets` is unused
+    const int32_t *seq_start, *seq_len, *lengths;
+    int anchor_back;
     float *out;      // [B, Hq, d]
     float *part;     // [U, gx, G, d + 2]: un-normalised output (block order), max, sum
     int span;        // rows per block, a multiple of 16
@@ -48,6 +52,23 @@ struct DecArgs {
     int native;      // 1: partials hold the mma tile order, 0: plain column order
     int32_t *dev_status;
 };
+
+// First row (in rows of head_dim elements from the array's start) and row count of unit u in K and in V.
+__device__ inline void unit_rows(const DecArgs &a, int u, int64_t &lo_k, int64_t &lo_v, int64_t &len64)
+{
+    if (!a.lengths) {
+        lo_k = lo_v = a.offsets[u];
+        len64 = a.offsets[u + 1] - lo_k;
+        return;
+    }
+    const int Hkv = a.p.num_kv_heads, s = u / Hkv, g = u % Hkv;
+    const int n = max(a.seq_len[s], 0);
+    const int b = max(0, min(a.lengths[u], n));
+    const int64_t first = (int64_t)a.seq_start[s] + (a.anchor_back ? n - b : 0);
+    lo_k = ((int64_t)s * a.p.k_stride_seq + (int64_t)g * a.p.k_stride_head) / a.p.head_dim + first;
+    lo_v = ((int64_t)s * a.p.v_stride_seq + (int64_t)g * a.p.v_stride_head) / a.p.head_dim + first;
+    len64 = b;
+}
 
 __device__ inline float dec_ex2(float x)
 {
@@ -165,8 +186,8 @@ decode_mma_kernel(DecArgs a)
     const int u = blockIdx.y, x = blockIdx.x, s = u / Hkv, g = u % Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = lane >> 2, c = lane & 3;
-    const int64_t lo = a.offsets[u];
-    const int64_t len64 = a.offsets[u + 1] - lo;
+    int64_t lo, lo_v, len64;
+    unit_rows(a, u, lo, lo_v, len64);
     const int len = (int)max((int64_t)0, min(len64, (int64_t)a.span * a.gx));
     if (len64 > len && x == 0 && threadIdx.x == 0 && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_CAPACITY);
     const int nblocks = ceil_div(len, a.span);
@@ -191,7 +212,7 @@ decode_mma_kernel(DecArgs a)
         }
     }
     const char *kbase = reinterpret_cast<const char *>(a.kc) + lo * D * 2;
-    const char *vbase = reinterpret_cast<const char *>(a.vc) + lo * D * 2;
+    const char *vbase = reinterpret_cast<const char *>(a.vc) + lo_v * D * 2;
 
     float o[NT][4];
 #pragma unroll
@@ -350,8 +371,8 @@ decode_lanes_kernel(DecArgs a)
     const int Hkv = p.num_kv_heads, G = p.num_q_heads / Hkv;
     const int u = blockIdx.y, x = blockIdx.x, s = u / Hkv, g = u % Hkv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t lo = a.offsets[u];
-    const int64_t len64 = a.offsets[u + 1] - lo;
+    int64_t lo, lo_v, len64;
+    unit_rows(a, u, lo, lo_v, len64);
     const int len = (int)max((int64_t)0, min(len64, (int64_t)a.span * a.gx));
     if (len64 > len && x == 0 && threadIdx.x == 0 && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_CAPACITY);
     const int nblocks = ceil_div(len, a.span);
@@ -364,7 +385,7 @@ decode_lanes_kernel(DecArgs a)
     const int begin = x * a.span, end = min(len, begin + a.span);
     const float scale = kLog2eDec * rsqrtf((float)D);
     const T *q = static_cast<const T *>(a.q) + ((int64_t)s * p.num_q_heads + g * G) * D;
-    const T *kc = static_cast<const T *>(a.kc) + lo * D, *vc = static_cast<const T *>(a.vc) + lo * D;
+    const T *kc = static_cast<const T *>(a.kc) + lo * D, *vc = static_cast<const T *>(a.vc) + lo_v * D;
     float qr[GMAX][E], o[GMAX][E], m[GMAX], l[GMAX];
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) {
@@ -420,7 +441,8 @@ decode_combine_kernel(DecArgs a)
     const refree_params &p = a.p;
     const int Hkv = p.num_kv_heads, G = p.num_q_heads / Hkv;
     const int u = blockIdx.x / G, h = blockIdx.x % G, s = u / Hkv, g = u % Hkv;
-    const int64_t len64 = a.offsets[u + 1] - a.offsets[u];
+    int64_t lo_k, lo_v, len64;
+    unit_rows(a, u, lo_k, lo_v, len64);
     const int len = (int)max((int64_t)0, min(len64, (int64_t)a.span * a.gx));
     const int nblocks = ceil_div(len, a.span);
     if (nblocks <= 1) return;                       // written by the attention kernel itself
@@ -510,12 +532,15 @@ size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows)
 
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,
                                     const int64_t *offsets, int64_t max_rows, float *out, void *workspace,
-                                    int32_t *dev_status, cudaStream_t st)
+                                    int32_t *dev_status, cudaStream_t st, const int32_t *seq_start,
+                                    const int32_t *seq_len, const int32_t *lengths, bool anchor_back)
 {
     DecArgs a;
     a.p = p;
     a.q = q_new; a.kc = k_c; a.vc = v_c;
     a.offsets = offsets;
+    a.seq_start = seq_start; a.seq_len = seq_len; a.lengths = lengths;
+    a.anchor_back = anchor_back ? 1 : 0;
     a.out = out;
     a.part = static_cast<float *>(workspace);
     a.dev_status = dev_status;

@@ -168,6 +168,8 @@ cudaError_t launch_compact_paged(const refree_params &p, const void *k, const vo
 size_t decode_workspace_bytes(const refree_params &p, int64_t max_rows);
 cudaError_t launch_decode_attention(const refree_params &p, const void *q_new, const void *k_c, const void *v_c,
                                     const int64_t *offsets, int64_t max_rows, float *out, void *workspace,
-                                    int32_t *dev_status, cudaStream_t st);
+                                    int32_t *dev_status, cudaStream_t st, const int32_t *seq_start = nullptr,
+                                    const int32_t *seq_len = nullptr, const int32_t *lengths = nullptr,
+                                    bool anchor_back = false);
 
 }  // namespace refree

@@ -100,6 +100,14 @@ def test_host_side_validation_of_the_layer_run_inplace_and_paged_entry_points(li
                                              binding.ANCHOR_BACK, fake, big, None, None) == binding.ERR_UNSUPPORTED
     assert lib.refree_compress_layer_inplace(ctypes.byref(c), fake, fake, fake, fake, fake, 128, fake, fake,
                                              binding.ANCHOR_BACK, None, 0, None, None) == binding.ERR_WORKSPACE
+    # decode over the in-place cache: token-major rows are not back to back
+    tm = binding.Params(1, 4, 2, 64, window=8, kv_tokens=128, k_strides=(0, 128, 64), v_strides=(0, 128, 64)).c_struct()
+    assert lib.refree_decode_attention_inplace(ctypes.byref(tm), fake, fake, fake, fake, fake, fake, binding.ANCHOR_BACK,
+                                               128, fake, fake, big, None, None) == binding.ERR_UNSUPPORTED
+    assert lib.refree_decode_attention_inplace(ctypes.byref(c), fake, fake, fake, fake, fake, None, binding.ANCHOR_BACK,
+                                               128, fake, fake, big, None, None) == binding.ERR_INVALID_ARG
+    assert lib.refree_decode_attention_inplace(ctypes.byref(c), fake, fake, fake, fake, fake, fake, binding.ANCHOR_BACK,
+                                               128, fake, None, 0, None, None) == binding.ERR_WORKSPACE
     # paged: block geometry, missing table, unaligned pool, score ranking without offsets
     assert lib.refree_compact_paged(ctypes.byref(c), fake, fake, fake, fake, fake, None, None, fake, 4, 0, fake, fake, 8,
                                     None, None) == binding.ERR_INVALID_ARG

@@ -197,6 +197,53 @@ def test_fused_inplace_pass_against_the_oracle(rank_mode, anchor, window, dtype)
             assert torch.equal(parity.bits(_unit_rows(vc, lay, s, g, b - a, back)), parity.bits(ref.v_out[a:b]))
 
 
+@pytest.mark.parametrize("anchor", [binding.ANCHOR_BACK, binding.ANCHOR_FRONT])
+@pytest.mark.parametrize("dtype,d,window", [("bf16", 128, 16), ("bf16", 64, 1), ("fp32", 128, 8)])
+def test_decode_step_over_the_cache_compacted_in_place(anchor, dtype, d, window):
+    """The in-place pass followed by one decode step that reads the strided ragged cache where it lies,
+    against the oracle's dense compaction followed by the oracle's decode attention."""
+    cfg = _cfg(window=window, dtype=dtype, head_dim=d, num_q_heads=8, num_kv_heads=2)
+    lay = workloads.make_layer(cfg, 5, seq_lens=[2500, 130, 0, 4097, 1])
+    p = binding.params_for(cfg, lay, threshold=0.05)
+    op = parity.oracle_params(p)
+    ref = orc.compress_layer(op, lay.q_win, lay.k, lay.v, lay.seq_start, lay.seq_len)
+    q_new = workloads.make_decode_query(cfg, 5, lay.q_win)
+    want = orc.decode_attention(op, q_new, ref.k_out, ref.v_out, ref.sel.offsets)
+    q, k, v, ss, sl = [t.to(DEV) for t in (lay.q_win, lay.k, lay.v, lay.seq_start, lay.seq_len)]
+    units = p.num_seqs * p.num_kv_heads
+    lengths = torch.zeros(units, dtype=torch.int32, device=DEV)
+    offsets = torch.zeros(units + 1, dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.empty(binding.refree_workspace_size(p, lay.total_tokens), dtype=torch.uint8, device=DEV)
+    binding.refree_compress_layer_inplace(p, q, k, v, ss, sl, lay.total_tokens, lengths, offsets, anchor, ws, status)
+    max_rows = int(lay.seq_len.max())
+    dws = torch.empty(binding.refree_decode_workspace_size(p, max_rows), dtype=torch.uint8, device=DEV)
+    out = torch.full((p.num_seqs, p.num_q_heads, d), float("nan"), dtype=torch.float32, device=DEV)
+    binding.refree_decode_attention_inplace(p, q_new.to(DEV), k, v, ss, sl, lengths, anchor, max_rows, out, dws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert lengths.cpu().tolist() == ref.sel.lengths.reshape(-1).tolist()
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    err = np.abs(got - want)
+    assert (err <= 1e-4 + 1e-4 * np.abs(want)).all(), float(err.max())
+    assert not got[2].any()                      # the empty sequence gives zero rows
+
+
+def test_decode_over_the_in_place_cache_needs_head_major_rows():
+    cfg = _cfg(window=8, dtype="bf16", head_dim=128, num_q_heads=4, num_kv_heads=2)
+    lay = workloads.make_layer(cfg, 0, layout="token_major", seq_lens=[100])
+    p = binding.params_for(cfg, lay)
+    k, v, ss, sl = [t.to(DEV) for t in (lay.k, lay.v, lay.seq_start, lay.seq_len)]
+    q_new = workloads.make_decode_query(cfg, 0, lay.q_win).to(DEV)
+    lengths = torch.full((2,), 50, dtype=torch.int32, device=DEV)
+    dws = torch.empty(binding.refree_decode_workspace_size(p, 100), dtype=torch.uint8, device=DEV)
+    out = torch.zeros(1, 4, 128, dtype=torch.float32, device=DEV)
+    rc = binding.refree_decode_attention_inplace(p, q_new, k, v, ss, sl, lengths, binding.ANCHOR_BACK, 100, out, dws,
+                                                 check=False)
+    assert rc == binding.ERR_UNSUPPORTED
+
+
 def test_inplace_flags_offsets_that_do_not_fit_the_sequences():
     cfg = _cfg(window=8, dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1)
     lay = workloads.make_layer(cfg, 0, seq_lens=[100])

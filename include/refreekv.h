@@ -230,8 +230,10 @@ refree_status refree_compress_layer_inplace(const refree_params *p, const void *
  * work is ordered after what `stream` holds at the call, and `stream` continues
  * only when every layer is done.  The first call on a device creates the two
  * internal streams (highest priority for scoring, lowest for compaction) and
- * their events, which live until the process exits; calls from several host
- * threads on one device share them and are serialised by stream order. */
+ * their events, which live until the process exits; the device that owns
+ * `stream` must be the current device of the calling thread.  Calls from
+ * several host threads on one device share the internal streams and are
+ * serialised by stream order. */
 refree_status refree_layers_workspace_size(const refree_params *p, int64_t total_tokens, size_t *bytes);
 refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
                                      const void *const *q_win, const void *const *k, const void *const *v,

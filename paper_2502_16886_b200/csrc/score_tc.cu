@@ -2,28 +2,34 @@
 //
 // The window logits S = Q K^T are the one dense contraction of the pass; they run
 // on tcgen05.mma with the accumulator in tensor memory, operands staged in shared
-// memory by TMA (128-byte swizzle).  A row's softmax normaliser needs all of the
-// row, and the column sums need every row's normaliser, so the logits are formed
-// twice (storing them would cost more HBM traffic than K itself):
+// memory by TMA (128-byte swizzle, no multicast).  A row's softmax normaliser needs
+// all of the row, and the column sums need every row's normaliser, so the logits are
+// formed twice (storing them would cost more HBM traffic than K itself):
 //
-//   pass 1  D[row, position] = Q_blk K_tile^T : one thread per query row sums
-//           2^(y - c) over the positions it may see (no cross-thread traffic);
-//           partial (c, Z) per (CTA, unit) go to the workspace
+//   pass 1  D[row, position] = Q_blk K_tile^T (M = 128 rows, N = 128 positions): one
+//           thread per query row sums 2^(y - c) over the positions it may see;
+//           partial (c, Z) per (CTA, unit, column half) go to the workspace
 //   pass 2  on entering a unit, L[row] = log2 sum_i 2^(y_i) is merged from those
-//           partials; then D[position, row] = K_tile Q^T : one thread per position
-//           sums 2^(y - L[row]) over the rows that see it -> a'[i]  (Eq. 2)
+//           partials; then D[position, row] = K_tile Q^T (M = 128 positions, N = up to
+//           256 rows in ONE product per k-step): one thread per position sums
+//           2^(y - L[row]) over the rows that see it -> a'[i]  (Eq. 2)
 //
-// Both passes use the same shared-memory images of Q and K (K-major, so either
-// can be the A or the B operand); only the roles swap, which puts each pass's
-// reduction inside a thread.  Persistent CTAs (one per SM) take contiguous ranges
-// of (unit, tile) items; warp 16 issues TMA, warp 17 issues MMA, warps 0-15 are the
-// epilogue: four warpgroups = (accumulator pair) x (64-column half of a 128-column
-// accumulator), two accumulators per pair in flight.  The exponentials bind, and with
-// four warps per scheduler instead of two their latencies overlap.  In pass 1 the two
-// halves of a row keep separate (c, Z) records; in pass 2 warpgroup 0 adds the other
-// warpgroups' column sums from shared memory.  Every wait is bounded: on a timeout the CTA records
-// REFREE_DEV_TIMEOUT, stops issuing work, and falls through to the common exit
-// where tensor memory is released.
+// Both passes use the same shared-memory images of Q and K (K-major, so either can be
+// the A or the B operand); only the roles swap, which puts each pass's reduction
+// inside a thread.  Measured on this part, consecutive products into one accumulator
+// cost about 137 cycles at N = 256 (93 % of the nominal rate) but 116-120 cycles at
+// N = 128 (55 %), and alternating between accumulators from one product to the next
+// is slower still; so pass 2 uses one wide product per k-step, and every accumulator
+// is handed back to the MMA warp as soon as its values sit in registers, before any
+// exponential is taken.
+//
+// Persistent CTAs (one per SM) take contiguous ranges of (unit, tile) items; warp 16
+// issues TMA, warp 17 issues MMA, warps 0-15 are the epilogue.  Pass 1: four
+// accumulators of 128 columns, warps = (accumulator pair) x (64-column half).  Pass 2:
+// two accumulators of 256 columns, warps = (lane quarter) x (column chunk); the warps of
+// chunk 0 add the other chunks' column sums from shared memory one tile late.  Every
+// wait is bounded: on a timeout the CTA records REFREE_DEV_TIMEOUT, stops issuing work,
+// and falls through to the common exit where tensor memory is released.
 #include <cuda.h>
 
 #include <algorithm>
@@ -35,8 +41,7 @@
 namespace refree {
 namespace {
 
-constexpr int kEpiWarps = 16;                 // four warpgroups: (accumulator pair) x (column half)
-constexpr int kHalfCols = 64;                 // tensor-memory columns of an accumulator per warpgroup
+constexpr int kEpiWarps = 16;
 constexpr int kThreadsTc = (kEpiWarps + 2) * 32;
 constexpr int kD = 128;
 constexpr int kHalfBytes = kTile * 128;          // one 64-column half of a 128-row tile: 16 KB
@@ -156,6 +161,10 @@ __device__ inline void tmem_ld_wait(uint32_t (&r)[32])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : RF_IO16(r, 0), RF_IO16(r, 16) :: "memory");
 }
+__device__ inline void tmem_ld_wait16(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : RF_IO16(r, 0) :: "memory");
+}
 __device__ inline float ex2(float x)
 {
     float y;
@@ -182,22 +191,44 @@ struct TcShape {
     int R;        // query rows per unit: G * window
     int Rpad;     // rows of the shared-memory Q image (multiple of 128)
     int rblocks;  // 128-row blocks: pass-1 accumulators per tile (A operands)
-    int cblocks;  // pass-2 accumulators per tile
-    int ncol;     // pass-2 columns (rows of Q) per accumulator: R / cblocks, at most 128
+    int cblocks;  // pass-2 products per k-step and tile: 1 up to 256 rows, else 2
+    int ncol;     // pass-2 columns (rows of Q) per product: a multiple of 16, cblocks * ncol >= R
     int stages;   // K tile ring depth
     int rank4;    // K tensor map has a sequence axis
 };
 
+// What the consumers of an item (one tile of one unit) need to know about it.  The TMA thread walks the
+// items and leaves one record per item in a ring in shared memory, written before the item's K tile is
+// requested; the MMA thread and the epilogue warps read it after the barriers that order them behind
+// that request, instead of each walking the item list in registers.
+struct ItemInfo {
+    int32_t u;        // unit = sequence * Hkv + head
+    int32_t g;        // KV head
+    int32_t n;        // length of the sequence
+    int32_t tile;     // tile index inside the sequence
+    int32_t ntiles;   // tiles of the sequence
+    int32_t pack;     // positions before the sequence in the packed score array
+    int32_t ib;       // index of the unit's first item
+    int32_t new_unit; // the item is the first of its unit in this CTA's pass
+};
+constexpr int kInfoRing = 16;   // the TMA thread runs at most ring stages + accumulators in flight ahead of the epilogue
+
 struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
-    uint64_t acc_full[4], acc_empty[4];       // accumulator (warpgroup * 2 + slot): 128 tensor-memory columns each
-    uint64_t half_ready[4];                   // pass 2: the other warpgroups have staged their shares of a tile
+    uint64_t acc_full[4], acc_empty[4];       // pass 1: accumulator (pair * 2 + slot), 128 tensor-memory columns each
+    uint64_t p2_full[2], p2_empty[2];         // pass 2: accumulators of 256 columns
+    uint64_t chunk_ready[4];                  // pass 2: the other column chunks have staged their shares of a tile
     uint32_t tmem_base;
     int abort_flag;
-    alignas(16) float stage[4][3][kTile];     // pass 2: partial column sums of warpgroups 1..3, four tiles deep
+    alignas(16) ItemInfo info[kInfoRing];
+    alignas(16) float stage[4][3][kTile];     // pass 2: partial column sums of chunks 1..3, four tiles deep
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
-    SeqTables seq;
-    int32_t start[kMaxSeqs];                  // copy of seq_start
+};
+
+// Per-sequence tables of the CTA behind the tail, sized by the number of sequences:
+// pack[B + 1], tiles[B + 1] (running sums of lengths and of tiles), len[B], start[B].
+struct SeqView {
+    const int32_t *pack, *tiles, *len, *start;
 };
 
 struct ItemTc {
@@ -205,36 +236,35 @@ struct ItemTc {
     int tile, ntiles;      // tile index inside the sequence, tiles of the sequence
 };
 
-__device__ inline void fill_seq_fields(ItemTc &it, const TcSmemTail &tl, int Hkv)
+__device__ inline void fill_seq_fields(ItemTc &it, const SeqView &sv, int Hkv)
 {
     it.u = it.s * Hkv + it.g;
-    it.n = tl.seq.len[it.s];
-    it.tok0 = tl.start[it.s];
-    it.pack = tl.seq.pack[it.s];
+    it.n = sv.len[it.s];
+    it.tok0 = sv.start[it.s];
+    it.pack = sv.pack[it.s];
     it.tile_start = it.tile * kTile;
 }
 
 // Items are ordered (sequence, head, tile): a CTA's consecutive items mostly share a unit.
-__device__ inline ItemTc decode_item_tc(const TcSmemTail &tl, int B, int Hkv, int item)
+__device__ inline ItemTc decode_item_tc(const SeqView &sv, int B, int Hkv, int item)
 {
-    const SeqTables &t = tl.seq;
     int lo = 0, hi = B;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if ((int64_t)t.tiles[mid] * Hkv <= item) lo = mid; else hi = mid;
+        if ((int64_t)sv.tiles[mid] * Hkv <= item) lo = mid; else hi = mid;
     }
     ItemTc it;
     it.s = lo;
-    it.ntiles = t.tiles[lo + 1] - t.tiles[lo];
-    const int rem = item - t.tiles[lo] * Hkv;
+    it.ntiles = sv.tiles[lo + 1] - sv.tiles[lo];
+    const int rem = item - sv.tiles[lo] * Hkv;
     it.g = rem / it.ntiles;
     it.tile = rem % it.ntiles;
-    fill_seq_fields(it, tl, Hkv);
+    fill_seq_fields(it, sv, Hkv);
     return it;
 }
 
 // The item after `it` in the same order, without searching or dividing.
-__device__ inline void next_item_tc(ItemTc &it, const TcSmemTail &tl, int B, int Hkv)
+__device__ inline void next_item_tc(ItemTc &it, const SeqView &sv, int B, int Hkv)
 {
     if (++it.tile < it.ntiles) {
         it.tile_start += kTile;
@@ -243,11 +273,11 @@ __device__ inline void next_item_tc(ItemTc &it, const TcSmemTail &tl, int B, int
     it.tile = 0;
     if (++it.g == Hkv) {
         it.g = 0;
-        do { ++it.s; } while (it.s < B - 1 && tl.seq.tiles[it.s + 1] == tl.seq.tiles[it.s]);
+        do { ++it.s; } while (it.s < B - 1 && sv.tiles[it.s + 1] == sv.tiles[it.s]);
         if (it.s >= B) it.s = B - 1;                 // past the end: never used, kept in range
-        it.ntiles = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
+        it.ntiles = sv.tiles[it.s + 1] - sv.tiles[it.s];
     }
-    fill_seq_fields(it, tl, Hkv);
+    fill_seq_fields(it, sv, Hkv);
 }
 
 // first item of CTA c when `items` are split evenly over `ctas`
@@ -259,8 +289,7 @@ struct TcArgs {
     const int32_t *seq_start, *seq_len;
     float2 *part;        // [2 (ctas + units)][Rpad]: one record per (CTA, unit, column half)
     GroupPartial *groups; // nullable: per 32 positions, exact sum of squared scores for the stopping rule
-    uint32_t *flags;     // fused launch: flags[c] == epoch once CTA c has written its pass-1 partials
-    uint32_t epoch;
+    uint32_t *flags;     // fused launch: flags[c] != 0 once CTA c has written its pass-1 partials (zeroed before the launch)
     float *scores;
     int64_t total_tokens;
     int32_t *dev_status;
@@ -277,27 +306,45 @@ __device__ inline bool epi_sync(TcSmemTail &tl, uint32_t &phase)
     return ok;
 }
 
-// Loop state that survives from pass 1 to pass 2 when both run in one launch.
-struct RingState { int stage = 0; uint32_t kphase = 0, qphase = 0; };
-struct MmaState : RingState { uint32_t cnt0 = 0, cnt1 = 0; int prev_u = -1; };
-struct EpiState { uint32_t cnt = 0, ephase = 0; };
+// Loop state that survives from pass 1 to pass 2 when both run in one launch.  `icount` numbers the
+// items a role has gone through in this launch (both passes): its low bits index the info ring.
+struct RingState { int stage = 0; uint32_t kphase = 0, qphase = 0, icount = 0; };
+struct MmaState : RingState { uint32_t cnt0 = 0, cnt1 = 0, cnt2 = 0; bool first = true; };
+struct EpiState { uint32_t ephase = 0, icount = 0; };
 
 // --------------------------------------------------------- producer / MMA -----
-template <int PASS>
 __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, const CUtensorMap *mapk,
-                                     unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
+                                     unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl, const SeqView &sv,
                                      int item0, int item1, RingState &rs)
 {
     const TcShape &sh = a.sh;
-    const int G = a.p.num_q_heads / a.p.num_kv_heads;
+    const int G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
     int cur_u = -1;
     int &stage = rs.stage;
     uint32_t &kphase = rs.kphase, &qphase = rs.qphase;
     bool ok = true;
     ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
-        if (it.u != cur_u) {
+    if (item0 < item1) it = decode_item_tc(sv, a.p.num_seqs, Hkv, item0);
+    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, sv, a.p.num_seqs, Hkv)) {
+        const bool new_unit = it.u != cur_u;
+        // the ring entry was last used sixteen items ago, which every consumer has long left behind
+        ItemInfo &inf = tl.info[rs.icount++ & (kInfoRing - 1)];
+        inf.u = it.u; inf.g = it.g; inf.n = it.n; inf.tile = it.tile; inf.ntiles = it.ntiles; inf.pack = it.pack;
+        inf.ib = sv.tiles[it.s] * Hkv + it.g * it.ntiles;
+        inf.new_unit = new_unit ? 1 : 0;
+        // The K tile first: the MMA thread learns of a unit change from the record, which it reads once
+        // the tile has landed, and only then gives the Q image back.
+        ok = mbar_wait(&tl.k_empty[stage], kphase ^ 1, &tl.abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(&tl.k_full[stage], (uint32_t)kTileBytes);     // (release) orders the record before the tile
+        unsigned char *dst = smem_k + (size_t)stage * kTileBytes;
+        for (int h = 0; h < 2; ++h) {
+            if (sh.rank4)
+                tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s);
+            else
+                tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g);
+        }
+        if (new_unit) {
             ok = mbar_wait(&tl.q_empty, qphase ^ 1, &tl.abort_flag);
             if (!ok) break;
             mbar_expect_tx(&tl.q_full, (uint32_t)sh.Rpad * 256u);
@@ -308,16 +355,6 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
                                 h * 64, row0 + rb * kTile);
             qphase ^= 1;
             cur_u = it.u;
-        }
-        ok = mbar_wait(&tl.k_empty[stage], kphase ^ 1, &tl.abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(&tl.k_full[stage], (uint32_t)kTileBytes);
-        unsigned char *dst = smem_k + (size_t)stage * kTileBytes;
-        for (int h = 0; h < 2; ++h) {
-            if (sh.rank4)
-                tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s);
-            else
-                tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g);
         }
         if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
     }
@@ -332,64 +369,108 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     }
 }
 
-// Accumulators: four of 128 tensor-memory columns.  Block b of a tile (a 128-row
-// block of Q in pass 1, a block of `ncol` rows of Q in pass 2) goes to warpgroup
-// b & 1, which owns two accumulators and alternates between them, so the MMA of a
-// warpgroup's next block runs while it reads the current one, and the two
-// warpgroups (hence the two warps sharing an SM sub-partition) drift out of phase.
-template <int PASS>
-__device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
-                                uint32_t tmem_base, int item0, int item1, MmaState &ms)
+// Pass 1.  Block b of a tile (a 128-row block of Q) goes to accumulator pair b & 1, which owns two
+// accumulators of 128 columns and alternates between them: the MMA of a pair's next block runs while
+// the epilogue reads the current one.
+__device__ inline void mma_loop_pass1(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
+                                      uint32_t tmem_base, int nitems, MmaState &ms)
 {
     const TcShape &sh = a.sh;
     const uint32_t q_lo = desc_lo(smem_u32(smem_q)), k_lo = desc_lo(smem_u32(smem_k));
     const uint32_t q_half = (uint32_t)(sh.Rpad * 128) >> 4;      // distance between the two 64-column halves of Q
-    const uint32_t idesc1 = make_idesc(kTile), idesc2 = make_idesc(sh.ncol);
-    const int blocks = PASS == 1 ? sh.rblocks : sh.cblocks;
-    int cur_u = -1;
-    int &stage = ms.stage, &prev_u = ms.prev_u;
-    uint32_t &kphase = ms.kphase, &qphase = ms.qphase, &cnt0 = ms.cnt0, &cnt1 = ms.cnt1;   // blocks issued per warpgroup
+    const uint32_t idesc = make_idesc(kTile);
+    int &stage = ms.stage;
+    uint32_t &kphase = ms.kphase, &qphase = ms.qphase, &cnt0 = ms.cnt0, &cnt1 = ms.cnt1;   // blocks issued per pair
     bool ok = true;
-    ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
-        if (it.u != cur_u) {
-            if (prev_u >= 0) umma_commit(&tl.q_empty);     // every MMA on the previous unit's Q has been issued
-            ok = mbar_wait(&tl.q_full, qphase, &tl.abort_flag);
-            if (!ok) break;
-            qphase ^= 1;
-            cur_u = it.u;
-            prev_u = it.u;
-        }
+    for (int item = 0; item < nitems && ok; ++item) {
         ok = mbar_wait(&tl.k_full[stage], kphase, &tl.abort_flag);
         if (!ok) break;
         tc_fence_after();
+        if (tl.info[ms.icount++ & (kInfoRing - 1)].new_unit) {
+            if (!ms.first) umma_commit(&tl.q_empty);       // every MMA on the previous unit's Q has been issued
+            ms.first = false;
+            ok = mbar_wait(&tl.q_full, qphase, &tl.abort_flag);
+            if (!ok) break;
+            qphase ^= 1;
+            tc_fence_after();
+        }
         const uint32_t kt_lo = k_lo + (uint32_t)stage * (kTileBytes >> 4);
-        for (int b = 0; b < blocks && ok; ++b) {
-            const int wg = b & 1;
-            const uint32_t cnt = wg ? cnt1 : cnt0;
-            const int acc = wg * 2 + (int)(cnt & 1u);
+        for (int b = 0; b < sh.rblocks && ok; ++b) {
+            const int pair = b & 1;
+            const uint32_t cnt = pair ? cnt1 : cnt0;
+            const int acc = pair * 2 + (int)(cnt & 1u);
             ok = mbar_wait(&tl.acc_empty[acc], ((cnt >> 1) & 1u) ^ 1u, &tl.abort_flag);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d0 = tmem_base + (uint32_t)acc * 128u;
-            if (PASS == 1) {
-                const uint32_t qa = q_lo + (uint32_t)b * (kHalfBytes >> 4);
+            const uint32_t qa = q_lo + (uint32_t)b * (kHalfBytes >> 4);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t h = kk >> 2, ko = (kk & 3) * 2;          // 32 bytes per K step of 16
-                    umma_bf16(d0, qa + h * q_half + ko, kt_lo + h * (kHalfBytes >> 4) + ko, kDescHi, idesc1, kk > 0);
-                }
-            } else {
-                const uint32_t qb = q_lo + (uint32_t)b * (uint32_t)(sh.ncol * 128 >> 4);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t h = kk >> 2, ko = (kk & 3) * 2;
-                    umma_bf16(d0, kt_lo + h * (kHalfBytes >> 4) + ko, qb + h * q_half + ko, kDescHi, idesc2, kk > 0);
-                }
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t h = kk >> 2, ko = (kk & 3) * 2;          // 32 bytes per K step of 16
+                umma_bf16(d0, qa + h * q_half + ko, kt_lo + h * (kHalfBytes >> 4) + ko, kDescHi, idesc, kk > 0);
             }
             umma_commit(&tl.acc_full[acc]);
-            if (wg) ++cnt1; else ++cnt0;
+            if (pair) ++cnt1; else ++cnt0;
+        }
+        umma_commit(&tl.k_empty[stage]);
+        if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
+    }
+}
+
+// The pass-2 accumulators (two of 256 columns) cover the same tensor-memory columns as the four of
+// pass 1: before the first pass-2 product, every pass-1 accumulator must have been handed back.
+__device__ inline bool drain_pass1(TcSmemTail &tl, const MmaState &ms)
+{
+    bool ok = true;
+    for (int pair = 0; pair < 2 && ok; ++pair) {
+        const uint32_t cnt = pair ? ms.cnt1 : ms.cnt0;
+        for (int slot = 0; slot < 2 && ok; ++slot) {
+            const uint32_t uses = (cnt + (slot ? 0u : 1u)) >> 1;
+            if (uses) ok = mbar_wait(&tl.acc_empty[pair * 2 + slot], (uses - 1u) & 1u, &tl.abort_flag);
+        }
+    }
+    if (ok) tc_fence_after();
+    return ok;
+}
+
+// Pass 2: D[position, row] = K_tile Q^T, `ncol` rows of Q per product.
+__device__ inline void mma_loop_pass2(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
+                                      uint32_t tmem_base, int nitems, MmaState &ms)
+{
+    const TcShape &sh = a.sh;
+    const uint32_t q_lo = desc_lo(smem_u32(smem_q)), k_lo = desc_lo(smem_u32(smem_k));
+    const uint32_t q_half = (uint32_t)(sh.Rpad * 128) >> 4;
+    const uint32_t idesc = make_idesc(sh.ncol);
+    int &stage = ms.stage;
+    uint32_t &kphase = ms.kphase, &qphase = ms.qphase, &cnt = ms.cnt2;
+    bool ok = true;
+    for (int item = 0; item < nitems && ok; ++item) {
+        ok = mbar_wait(&tl.k_full[stage], kphase, &tl.abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (tl.info[ms.icount++ & (kInfoRing - 1)].new_unit) {
+            if (!ms.first) umma_commit(&tl.q_empty);
+            ms.first = false;
+            ok = mbar_wait(&tl.q_full, qphase, &tl.abort_flag);
+            if (!ok) break;
+            qphase ^= 1;
+            tc_fence_after();
+        }
+        const uint32_t kt_lo = k_lo + (uint32_t)stage * (kTileBytes >> 4);
+        for (int cb = 0; cb < sh.cblocks && ok; ++cb) {
+            const int buf = (int)(cnt & 1u);
+            ok = mbar_wait(&tl.p2_empty[buf], ((cnt >> 1) & 1u) ^ 1u, &tl.abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d0 = tmem_base + (uint32_t)buf * 256u;
+            const uint32_t qb = q_lo + (uint32_t)cb * (uint32_t)(sh.ncol * 128 >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t h = kk >> 2, ko = (kk & 3) * 2;
+                umma_bf16(d0, kt_lo + h * (kHalfBytes >> 4) + ko, qb + h * q_half + ko, kDescHi, idesc, kk > 0);
+            }
+            umma_commit(&tl.p2_full[buf]);
+            ++cnt;
         }
         umma_commit(&tl.k_empty[stage]);
         if (++stage == sh.stages) { stage = 0; kphase ^= 1; }
@@ -397,19 +478,15 @@ __device__ inline void mma_loop(const TcArgs &a, unsigned char *smem_q, unsigned
 }
 
 // ------------------------------------------------------------- epilogues -----
-// Pass 1: thread = query row.  Sum of 2^(y - c) over the positions the row sees.
+// Pass 1: thread = query row, 64 logits of the row in registers.
 template <bool MASKED>
-__device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, int limit)
+__device__ inline float row_sum_regs(const uint32_t (&ra)[32], const uint32_t (&rb)[32], float scale, float cref, int limit)
 {
     float z0 = 0.f, z1 = 0.f;
     const float nc = -cref;
-    uint32_t ra[32], rb[32];
-    tmem_ld32_issue(taddr, ra);
-    tmem_ld32_issue(taddr + 32, rb);
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-        uint32_t (&cur)[32] = c ? rb : ra;
-        tmem_ld_wait(cur);
+        const uint32_t (&cur)[32] = c ? rb : ra;
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
             float e0 = ex2(fmaf(__uint_as_float(cur[i]), scale, nc));
@@ -424,16 +501,12 @@ __device__ inline float row_sum_tile(uint32_t taddr, float scale, float cref, in
     }
     return z0 + z1;
 }
-__device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
+__device__ inline float row_max_regs(const uint32_t (&ra)[32], const uint32_t (&rb)[32], float scale, int limit)
 {
     float m = -INFINITY;
-    uint32_t ra[32], rb[32];
-    tmem_ld32_issue(taddr, ra);
-    tmem_ld32_issue(taddr + 32, rb);
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-        uint32_t (&cur)[32] = c ? rb : ra;
-        tmem_ld_wait(cur);
+        const uint32_t (&cur)[32] = c ? rb : ra;
 #pragma unroll
         for (int i = 0; i < 32; ++i)
             if (c * 32 + i < limit) m = fmaxf(m, __uint_as_float(cur[i]) * scale);
@@ -441,23 +514,22 @@ __device__ inline float row_max_tile(uint32_t taddr, float scale, int limit)
     return m;
 }
 
-__device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1,
-                                      EpiState &es)
+__device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int nitems, EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int wg = (warp >> 2) & 1, half = warp >> 3, lane_base = (warp & 3) * 32;
+    const int pair = (warp >> 2) & 1, half = warp >> 3, lane_base = (warp & 3) * 32;
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
     int cur_u = -1;
-    uint32_t &cnt = es.cnt;                      // blocks this warpgroup has consumed
-    // running reference and sum of this thread's rows (row blocks wg and wg + 2) over its half of the columns
+    uint32_t cnt = 0;                            // blocks this accumulator pair has consumed
+    // running reference and sum of this thread's rows (row blocks pair and pair + 2) over its half of the columns
     float cref[2] = {-INFINITY, -INFINITY}, zsum[2] = {0.f, 0.f};
     int rmod[2];
     bool rvalid[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-        const int row = (wg + 2 * j) * kTile + lane_base + lane;
+        const int row = (pair + 2 * j) * kTile + lane_base + lane;
         rmod[j] = row % w;                       // offset of the row's query inside the window
         rvalid[j] = row < sh.R;
     }
@@ -465,7 +537,7 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
     auto flush = [&](int u) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            const int rb = wg + 2 * j;
+            const int rb = pair + 2 * j;
             const int row = rb * kTile + lane_base + lane;
             if (rb < sh.rblocks && row < sh.R)
                 a.part[((int64_t)(blockIdx.x + u) * 2 + half) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
@@ -473,100 +545,139 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             zsum[j] = 0.f;
         }
     };
-    ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, a.p.num_kv_heads, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, a.p.num_kv_heads)) {
-        if (it.u != cur_u) {
-            if (cur_u >= 0) flush(cur_u);
-            cur_u = it.u;
-        }
+    for (int item = 0; item < nitems && ok; ++item) {
+        const ItemInfo *inf = &tl.info[es.icount++ & (kInfoRing - 1)];
+        int tile_start = 0, n = 0;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            const int rb = wg + 2 * j;
+            const int rb = pair + 2 * j;
             if (rb >= sh.rblocks || !ok) continue;
-            const int acc = wg * 2 + (int)(cnt & 1u);
+            const int acc = pair * 2 + (int)(cnt & 1u);
             ok = mbar_wait(&tl.acc_full[acc], (cnt >> 1) & 1u, &tl.abort_flag);
             if (!ok) continue;
             ++cnt;
             tc_fence_after();
+            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + (uint32_t)(half * 64) + ((uint32_t)lane_base << 16);
+            uint32_t ra[32], rb2[32];
+            tmem_ld32_issue(taddr, ra);
+            tmem_ld32_issue(taddr + 32, rb2);
+            tmem_ld_wait(ra);
+            tmem_ld_wait(rb2);
+            // the logits are in registers: the accumulator goes back to the MMA warp before any arithmetic
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
+            if (j == 0 || sh.rblocks <= 2) {
+                // the item's record is valid from the first accumulator of the item on
+                const int u = inf->u;
+                if (u != cur_u) {
+                    if (cur_u >= 0) flush(cur_u);
+                    cur_u = u;
+                }
+                tile_start = inf->tile * kTile;
+                n = inf->n;
+            }
+            const bool full = tile_start + kTile <= n - w + 1;      // tile wholly before the window
             int limit = kTile;                                  // visible positions of the tile: [0, limit)
-            const bool full = it.tile_start + kTile <= it.n - w + 1;   // tile wholly before the window
             if (!full) {
-                limit = it.n - w + rmod[j] - it.tile_start + 1;     // up to this row's own position
-                limit = (rvalid[j]) ? max(0, min(kTile, limit)) : 0;
+                limit = n - w + rmod[j] - tile_start + 1;           // up to this row's own position
+                limit = rvalid[j] ? max(0, min(kTile, limit)) : 0;
             } else if (!rvalid[j]) {
                 limit = 0;
             }
-            limit = max(0, min(kHalfCols, limit - half * kHalfCols));   // inside this warpgroup's columns
-            const bool uniform = __all_sync(0xffffffffu, limit == kHalfCols);
-            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + (uint32_t)(half * kHalfCols) + ((uint32_t)lane_base << 16);
+            limit = max(0, min(64, limit - half * 64));         // inside this warp's columns
+            const bool uniform = __all_sync(0xffffffffu, limit == 64);
             bool need_max = (cref[j] == -INFINITY) && limit > 0;
             float zt = 0.f;
             for (int attempt = 0; attempt < 2; ++attempt) {
                 if (__any_sync(0xffffffffu, need_max)) {
-                    const float m = row_max_tile(taddr, scale, limit);
+                    const float m = row_max_regs(ra, rb2, scale, limit);
                     if (need_max && m > cref[j]) {
                         zsum[j] = (cref[j] == -INFINITY) ? 0.f : zsum[j] * ex2(cref[j] - m);
                         cref[j] = m;
                     }
                 }
-                zt = uniform ? row_sum_tile<false>(taddr, scale, cref[j], limit)
-                             : row_sum_tile<true>(taddr, scale, cref[j], limit);
+                zt = uniform ? row_sum_regs<false>(ra, rb2, scale, cref[j], limit)
+                             : row_sum_regs<true>(ra, rb2, scale, cref[j], limit);
                 need_max = !(zt <= kZLimit) && limit > 0;       // overflow against a stale reference
                 if (attempt == 1 || !__any_sync(0xffffffffu, need_max)) break;
             }
             if (limit > 0) zsum[j] += zt;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
         }
     }
     if (cur_u >= 0 && ok) flush(cur_u);
 }
 
-// Pass 2: thread = position.  Sum over the rows that see it of 2^(y - L[row]).
-// One accumulator's share of a warpgroup: ncol_wg columns (a multiple of 16, at most
-// 64) in two chunks of up to 32, both loads in flight.
+// Pass 2: thread = position.  One product's share of a warp: WIDTH columns (rows of Q; 16, 32, 48 or 64) come
+// from tensor memory 16 at a time, the next 16 in flight while 2^(y - L[row]) is summed over the current ones;
+// the accumulator is handed back as soon as the last load has landed.
+// rbase = row of the first column; pos_gap = i - (n - w): row r sees position i iff (r mod w) >= pos_gap.
 template <bool MASKED>
-__device__ inline float col_sum_job(uint32_t taddr, float scale, const float *lse, int rbase, int ncol_wg,
-                                    int w, int pos_gap)
+__device__ inline void col_sum16(const uint32_t (&cur)[32], float scale, const float *lse, int r0, int R, int w,
+                                 int pos_gap, float &s0, float &s1)
 {
-    // pos_gap = i - (n - w): row r sees position i iff (r mod w) >= pos_gap
-    uint32_t ra[32] = {}, rb[32] = {};
-    float s0 = 0.f, s1 = 0.f;
-    if (ncol_wg >= 32) tmem_ld32_issue(taddr, ra); else tmem_ld16_issue(taddr, ra);
-    if (ncol_wg >= 64) tmem_ld32_issue(taddr + 32, rb); else if (ncol_wg > 32) tmem_ld16_issue(taddr + 32, rb);
+    int rloc = MASKED ? r0 % w : 0;
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
-        if (c * 32 < ncol_wg) {
-            uint32_t (&cur)[32] = c ? rb : ra;
-            tmem_ld_wait(cur);
-            const int r0 = rbase + c * 32;
-            const int width = min(32, ncol_wg - c * 32);
-            int rloc = MASKED ? r0 % w : 0;
+    for (int i = 0; i < 16; i += 4) {
+        const float4 L = *reinterpret_cast<const float4 *>(lse + r0 + i);
+        float e[4];
+        e[0] = ex2(fmaf(__uint_as_float(cur[i]), scale, -L.x));
+        e[1] = ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -L.y));
+        e[2] = ex2(fmaf(__uint_as_float(cur[i + 2]), scale, -L.z));
+        e[3] = ex2(fmaf(__uint_as_float(cur[i + 3]), scale, -L.w));
+        if (MASKED) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                if (i < width) {
-                    const float4 L = *reinterpret_cast<const float4 *>(lse + r0 + i);
-                    float e[4];
-                    e[0] = ex2(fmaf(__uint_as_float(cur[i]), scale, -L.x));
-                    e[1] = ex2(fmaf(__uint_as_float(cur[i + 1]), scale, -L.y));
-                    e[2] = ex2(fmaf(__uint_as_float(cur[i + 2]), scale, -L.z));
-                    e[3] = ex2(fmaf(__uint_as_float(cur[i + 3]), scale, -L.w));
-                    if (MASKED) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if (rloc < pos_gap) e[j] = 0.f;
-                            if (++rloc == w) rloc = 0;
-                        }
-                    }
-                    s0 += e[0] + e[2];
-                    s1 += e[1] + e[3];
-                }
+            for (int j = 0; j < 4; ++j) {
+                if (rloc < pos_gap || r0 + i + j >= R) e[j] = 0.f;     // hidden by causality, or padding
+                if (++rloc == w) rloc = 0;
             }
         }
+        s0 += e[0] + e[2];
+        s1 += e[1] + e[3];
+    }
+}
+
+template <int WIDTH, bool MASKED>
+__device__ inline float col_job(uint32_t taddr, uint64_t *empty_bar, int lane, float scale, const float *lse,
+                                int rbase, int R, int w, int pos_gap)
+{
+    constexpr int NCH = WIDTH / 16;
+    uint32_t b0[32], b1[32];               // only the first 16 of each are used
+    float s0 = 0.f, s1 = 0.f;
+    tmem_ld16_issue(taddr, b0);
+    tmem_ld_wait16(b0);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        uint32_t (&cur)[32] = (c & 1) ? b1 : b0;
+        uint32_t (&nxt)[32] = (c & 1) ? b0 : b1;
+        if (c + 1 < NCH) tmem_ld16_issue(taddr + 16 * (c + 1), nxt);
+        if (c + 1 == NCH) {
+            // every load has landed
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar);
+        }
+        col_sum16<MASKED>(cur, scale, lse, rbase + 16 * c, R, w, pos_gap, s0, s1);
+        if (c + 1 < NCH) tmem_ld_wait16(nxt);
     }
     return s0 + s1;
+}
+
+template <bool MASKED>
+__device__ inline float col_job_any(int width, uint32_t taddr, uint64_t *empty_bar, int lane, float scale,
+                                    const float *lse, int rbase, int R, int w, int pos_gap)
+{
+    switch (width) {
+    case 64: return col_job<64, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
+    case 48: return col_job<48, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
+    case 32: return col_job<32, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
+    case 16: return col_job<16, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
+    default:
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar);
+        return 0.f;
+    }
 }
 
 // CTA that owns item x when `items` are split evenly over `ctas` (ctas <= items).
@@ -575,146 +686,160 @@ __device__ inline int cta_of_item(int x, int items, int ctas)
     return (int)((((int64_t)x + 1) * ctas - 1) / items);
 }
 
-__device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, uint32_t tmem_base, int item0, int item1,
-                                      int items, int ctas, EpiState &es)
+__device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const SeqView &sv, uint32_t tmem_base,
+                                      int nitems, int items, int ctas, EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int grp = warp >> 2;                                     // 0 finishes the tile, 1..3 stage their shares
-    const int wg = grp & 1, half = grp >> 1, lane_base = (warp & 3) * 32;
+    const int chunk = warp >> 2;                                   // 0 finishes the tile, 1..3 stage their shares
+    const int lane_base = (warp & 3) * 32;
     const int tid = threadIdx.x;                                   // 0..511
     const float scale = kLog2e * rsqrtf((float)kD);
-    const int w = a.p.window, G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
+    const int w = a.p.window;
     const int pos_in_tile = lane_base + lane;
-    const bool two_halves = sh.cblocks > 1;                        // both warpgroups contribute to a tile
-    int cur_u = -1;
-    uint32_t &cnt = es.cnt, &ephase = es.ephase;                   // blocks consumed, phase of the epilogue barrier
+    // this warp's columns of a product: whole groups of 16, split as evenly as the four chunks allow
+    const int units16 = sh.ncol >> 4;
+    const int c_begin = (chunk * units16 / 4) * 16, c_width = ((chunk + 1) * units16 / 4) * 16 - c_begin;
+    const bool exact = sh.cblocks * sh.ncol == sh.R;               // no padding columns in the products
+    uint32_t cnt = 0;                                              // products consumed
+    uint32_t &ephase = es.ephase;                                  // phase of the epilogue barrier
     uint32_t tcount = 0;                                           // tiles seen
-    // warpgroup 0 finishes a tile one tile late, when the other warpgroups' shares have long been staged
-    float pend_acc = 0.f, pend_norm = 0.f;
-    float *pend_dst = nullptr;
-    GroupPartial *pend_grp = nullptr;
-    uint32_t pend_tile = 0;
-    bool pending = false, ok = true;
+    // chunk 0 finishes a tile one tile late, when the other chunks' shares have long been staged
+    float pend_acc = 0.f;
+    const ItemInfo *pend_inf = nullptr;        // the pending tile's record (still in the ring: it is one item old)
+    bool ok = true;
     auto finish_pending = [&]() -> bool {
-        if (!pending) return true;
+        if (!pend_inf) return true;
+        const uint32_t pend_tile = tcount - 1u;
         float tot = pend_acc;
-        if (!mbar_wait(&tl.half_ready[pend_tile & 3u], (pend_tile >> 2) & 1u, &tl.abort_flag)) return false;
-        tot += tl.stage[pend_tile & 3u][1][pos_in_tile];                       // same accumulators, other columns
-        if (two_halves) tot += tl.stage[pend_tile & 3u][0][pos_in_tile] + tl.stage[pend_tile & 3u][2][pos_in_tile];
+        if (!mbar_wait(&tl.chunk_ready[pend_tile & 3u], (pend_tile >> 2) & 1u, &tl.abort_flag)) return false;
+        tot += tl.stage[pend_tile & 3u][0][pos_in_tile];
+        tot += tl.stage[pend_tile & 3u][1][pos_in_tile];
+        tot += tl.stage[pend_tile & 3u][2][pos_in_tile];
+        const int n = pend_inf->n, i = pend_inf->tile * kTile + pos_in_tile;
+        const int G = a.p.num_q_heads / a.p.num_kv_heads;
+        const int cnt_i = max(1, min(min(w, n), n - i));
         float sc = 0.f;
-        if (pend_dst) {
-            sc = tot * pend_norm;
+        if (i < n) {
+            sc = tot / ((float)cnt_i * (float)G);
             if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
-            *pend_dst = sc;
+            a.scores[(int64_t)pend_inf->g * a.total_tokens + pend_inf->pack + i] = sc;
         }
-        if (pend_grp) {
+        if (a.groups) {
             // this warp's 32 positions: largest score, and the exact squares summed at a scale set by it
-            const uint32_t bits = (pend_dst && isfinite(sc)) ? mag_bits(sc) : 0u;
+            const uint32_t bits = (i < n && isfinite(sc)) ? mag_bits(sc) : 0u;
             const uint32_t mx = __reduce_max_sync(0xffffffffu, bits);
             unsigned long long sq = sq_fixed(bits, kGroupShift - 2 * max(1, (int)(mx >> 23)));
             for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-            if (lane == 0) { GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq; *pend_grp = gp; }
+            if (lane == 0) {
+                GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq;
+                a.groups[((int64_t)pend_inf->ib + pend_inf->tile) * 4 + (warp & 3)] = gp;
+            }
         }
-        pending = false;
+        pend_inf = nullptr;
         return true;
     };
-    ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(tl, a.p.num_seqs, Hkv, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, tl, a.p.num_seqs, Hkv)) {
-        if (it.u != cur_u) {
-            if (!(ok = epi_sync(tl, ephase))) break;               // nobody still reads the previous unit's L
-            // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
-            // left per (CTA, unit), in ascending CTA order (the same order in every CTA that needs it)
-            const int ts = tl.seq.tiles[it.s + 1] - tl.seq.tiles[it.s];
-            const int ib = tl.seq.tiles[it.s] * Hkv + it.g * ts;
-            const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
-            if (a.flags) {
-                // one launch for both passes: the partials of this unit come from CTAs that may still be in
-                // pass 1; wait (bounded) until each of them has published
-                for (int c = c_lo + tid; c <= c_hi; c += kEpiWarps * 32) {
-                    bool seen = false;
-                    for (uint32_t spin = 0; spin < kSpinLimit && !seen; ++spin) {
-                        uint32_t v;
-                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.flags + c) : "memory");
-                        seen = v == a.epoch;
-                        if (!seen) { if (tl.abort_flag) break; __nanosleep(spin > 64 ? 256 : 32); }
-                    }
-                    if (!seen) tl.abort_flag = 1;
-                }
-                if (!(ok = epi_sync(tl, ephase))) break;
-                if (tl.abort_flag) { ok = false; break; }
-            }
-            for (int r = tid; r < sh.R; r += kEpiWarps * 32) {
-                float M = -INFINITY, Z = 0.f;
-                const int s_hi = 2 * (c_hi + it.u) + 1;             // records: (CTA, column half)
-                for (int s0 = 2 * (c_lo + it.u); s0 <= s_hi; s0 += 8) {
-                    float2 pr[8];                                  // eight independent loads in flight
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        pr[q] = (s0 + q <= s_hi) ? __ldcg(&a.part[(int64_t)(s0 + q) * sh.Rpad + r])
-                                                 : make_float2(-INFINITY, 0.f);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (pr[q].y > 0.f) {
-                            if (pr[q].x > M) { Z = Z * ex2(M - pr[q].x) + pr[q].y; M = pr[q].x; }
-                            else Z += pr[q].y * ex2(pr[q].x - M);
-                        }
-                    }
-                }
-                tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;     // a row that sees nothing adds 2^(-inf) = 0
-            }
-            if (!(ok = epi_sync(tl, ephase))) break;
-            cur_u = it.u;
-        }
-        const int i = it.tile_start + pos_in_tile;
-        const int pos_gap = i - (it.n - w);
-        // tile wholly before the window and wholly inside the sequence: every row sees every position
-        const bool full = it.tile_start + kTile <= it.n - w + 1;
+    for (int item = 0; item < nitems && ok; ++item) {
+        const ItemInfo *inf = &tl.info[es.icount++ & (kInfoRing - 1)];
         float accv = 0.f;
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int cb = wg + 2 * j;
-            if (cb >= sh.cblocks || !ok) continue;
-            const int acc = wg * 2 + (int)(cnt & 1u);
-            ok = mbar_wait(&tl.acc_full[acc], (cnt >> 1) & 1u, &tl.abort_flag);
-            if (!ok) continue;
+        int tile_start = 0, n = 0;
+        for (int cb = 0; cb < sh.cblocks && ok; ++cb) {
+            const int buf = (int)(cnt & 1u);
+            ok = mbar_wait(&tl.p2_full[buf], (cnt >> 1) & 1u, &tl.abort_flag);
+            if (!ok) break;
             ++cnt;
             tc_fence_after();
-            const int c_off = half * kHalfCols, ncol_h = max(0, min(kHalfCols, sh.ncol - c_off));
-            const uint32_t taddr = tmem_base + (uint32_t)acc * 128u + (uint32_t)c_off + ((uint32_t)lane_base << 16);
-            if (ncol_h > 0)
-                accv += full ? col_sum_job<false>(taddr, scale, tl.lse, cb * sh.ncol + c_off, ncol_h, w, pos_gap)
-                             : col_sum_job<true>(taddr, scale, tl.lse, cb * sh.ncol + c_off, ncol_h, w, pos_gap);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.acc_empty[acc]);
+            if (cb == 0) {
+                // the item's record is valid from the item's first product on
+                if (inf->new_unit) {
+                    if (!(ok = epi_sync(tl, ephase))) break;       // nobody still reads the previous unit's L
+                    // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
+                    // left per (CTA, unit), in ascending CTA order (the same order in every CTA that needs it)
+                    const int u = inf->u, ts = inf->ntiles, ib = inf->ib;
+                    const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
+                    if (a.flags) {
+                        // one launch for both passes: the partials of this unit come from CTAs that may still be
+                        // in pass 1; wait (bounded) until each of them has published
+                        for (int c = c_lo + tid; c <= c_hi; c += kEpiWarps * 32) {
+                            bool seen = false;
+                            for (uint32_t spin = 0; spin < kSpinLimit && !seen; ++spin) {
+                                uint32_t v;
+                                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.flags + c) : "memory");
+                                seen = v != 0u;
+                                if (!seen) { if (tl.abort_flag) break; __nanosleep(spin > 64 ? 256 : 32); }
+                            }
+                            if (!seen) tl.abort_flag = 1;
+                        }
+                        if (!(ok = epi_sync(tl, ephase))) break;
+                        if (tl.abort_flag) { ok = false; break; }
+                    }
+                    // two threads per row when there are enough threads: even and odd records, then one exchange
+                    const int per_row = 2 * sh.R <= kEpiWarps * 32 ? 2 : 1;
+                    const int r = tid / per_row, sub = tid % per_row;
+                    float M = -INFINITY, Z = 0.f;
+                    if (r < sh.R) {
+                        const int s_hi = 2 * (c_hi + u) + 1;               // records: (CTA, column half)
+                        for (int s0 = 2 * (c_lo + u) + sub; s0 <= s_hi; s0 += 8 * per_row) {
+                            float2 pr[8];                                  // eight independent loads in flight
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                pr[q] = (s0 + q * per_row <= s_hi)
+                                            ? __ldcg(&a.part[(int64_t)(s0 + q * per_row) * sh.Rpad + r])
+                                            : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                if (pr[q].y > 0.f) {
+                                    if (pr[q].x > M) { Z = Z * ex2(M - pr[q].x) + pr[q].y; M = pr[q].x; }
+                                    else Z += pr[q].y * ex2(pr[q].x - M);
+                                }
+                            }
+                        }
+                    }
+                    if (per_row == 2) {
+                        const float M2 = __shfl_xor_sync(0xffffffffu, M, 1), Z2 = __shfl_xor_sync(0xffffffffu, Z, 1);
+                        // (even records) then (odd records), in that order on both lanes
+                        const float Ma = sub ? M2 : M, Za = sub ? Z2 : Z, Mb = sub ? M : M2, Zb = sub ? Z : Z2;
+                        if (Zb > 0.f) {
+                            if (Za > 0.f) {
+                                if (Mb > Ma) { Z = Za * ex2(Ma - Mb) + Zb; M = Mb; }
+                                else { Z = Za + Zb * ex2(Mb - Ma); M = Ma; }
+                            } else { Z = Zb; M = Mb; }
+                        } else { Z = Za; M = Ma; }
+                    }
+                    // a row that sees nothing adds 2^(-inf) = 0
+                    if (r < sh.R && sub == 0) tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;
+                    // columns past the unit's rows (padding of the last product) never count
+                    for (int rr = sh.R + tid; rr < sh.cblocks * sh.ncol; rr += kEpiWarps * 32) tl.lse[rr] = INFINITY;
+                    if (!(ok = epi_sync(tl, ephase))) break;
+                }
+                tile_start = inf->tile * kTile;
+                n = inf->n;
+            }
+            const int pos_gap = tile_start + pos_in_tile - (n - w);
+            // tile wholly before the window and wholly inside the sequence: every row sees every position
+            const bool full = tile_start + kTile <= n - w + 1 && exact;
+            const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)c_begin + ((uint32_t)lane_base << 16);
+            accv += full ? col_job_any<false>(c_width, taddr, &tl.p2_empty[buf], lane, scale, tl.lse, cb * sh.ncol + c_begin,
+                                              sh.R, w, pos_gap)
+                         : col_job_any<true>(c_width, taddr, &tl.p2_empty[buf], lane, scale, tl.lse, cb * sh.ncol + c_begin,
+                                             sh.R, w, pos_gap);
         }
         if (!ok) break;
-        // Warpgroup 0 completes the previous tile only now, after it has handed this tile's accumulators
-        // back, so the MMA of the tile after next overlaps the completion.  The others can then be at most
-        // three tiles past the staging slot read here (the accumulators of tile t + 3 need this warpgroup's
-        // release of tile t + 1, which comes after this point): four slots.
-        if (grp == 0 && !(ok = finish_pending())) break;
-        if (grp == 0) {
-            const int cnt_i = max(1, min(min(w, it.n), it.n - i));
+        // Chunk 0 completes the previous tile only now, so its wait for the other chunks' shares of that
+        // tile has long been satisfied.  The others can be at most three tiles past the staging slot read
+        // here (an accumulator is handed back by all sixteen warps, chunk 0 included): four slots.
+        if (chunk == 0) {
+            if (!(ok = finish_pending())) break;
             pend_acc = accv;
-            pend_norm = 1.f / ((float)cnt_i * (float)G);
-            pend_dst = i < it.n ? a.scores + (int64_t)it.g * a.total_tokens + it.pack + i : nullptr;
-            pend_grp = a.groups ? a.groups + ((int64_t)tl.seq.tiles[it.s] * Hkv + (int64_t)it.g * it.ntiles + it.tile) * 4 +
-                                      (warp & 3)
-                                : nullptr;
-            pend_tile = tcount;
-            pending = true;
-        } else if (wg == 0 || two_halves) {
-            // the second accumulator pair has blocks (and is paced by the MMA warp) only with several column blocks
-            tl.stage[tcount & 3u][grp - 1][pos_in_tile] = accv;
+            pend_inf = inf;
+        } else {
+            tl.stage[tcount & 3u][chunk - 1][pos_in_tile] = accv;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.half_ready[tcount & 3u]);
+            if (lane == 0) mbar_arrive(&tl.chunk_ready[tcount & 3u]);
         }
         ++tcount;
     }
-    if (grp == 0 && ok) finish_pending();
+    if (chunk == 0 && ok) finish_pending();
 }
 
 // ---------------------------------------------------------------- kernels ----
@@ -728,6 +853,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     unsigned char *smem_q = smem;
     unsigned char *smem_k = smem + (size_t)sh.Rpad * 256;
     TcSmemTail &tl = *reinterpret_cast<TcSmemTail *>(smem_k + (size_t)sh.stages * kTileBytes);
+    int32_t *tab = reinterpret_cast<int32_t *>(&tl + 1);
+    const int B = a.p.num_seqs;
+    int32_t *t_pack = tab, *t_tiles = tab + (B + 1), *t_len = tab + 2 * (B + 1), *t_start = tab + 2 * (B + 1) + B;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == kEpiWarps * 32) {
@@ -739,22 +867,36 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         mbar_init(&tl.q_full, 1);
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
-        // stagers: the other column half of the first accumulator pair, plus both halves of the second pair
-        for (int b = 0; b < 4; ++b) mbar_init(&tl.half_ready[b], a.sh.cblocks > 1 ? 12 : 4);
+        for (int b = 0; b < 2; ++b) { mbar_init(&tl.p2_full[b], 1); mbar_init(&tl.p2_empty[b], kEpiWarps); }
+        for (int b = 0; b < 4; ++b) mbar_init(&tl.chunk_ready[b], 12);      // the twelve warps of chunks 1..3
         mbar_init(&tl.epi_bar, kEpiWarps);
         tl.abort_flag = 0;
         fence_barrier_init();
     }
-    for (int t = threadIdx.x; t < a.p.num_seqs; t += kThreadsTc) tl.start[t] = a.seq_start[t];
-    build_seq_tables(tl.seq, a.seq_len, a.p.num_seqs);       // ends with __syncthreads()
+    for (int t = threadIdx.x; t < B; t += kThreadsTc) t_start[t] = a.seq_start[t];
+    if (threadIdx.x == 32) {
+        int32_t pa = 0, ti = 0;
+        for (int s = 0; s < B; ++s) {
+            t_pack[s] = pa;
+            t_tiles[s] = ti;
+            const int n = max(a.seq_len[s], 0);
+            t_len[s] = n;
+            pa += n;
+            ti += ceil_div(n, kTile);
+        }
+        t_pack[B] = pa;
+        t_tiles[B] = ti;
+    }
     if (warp == kEpiWarps + 1) tmem_alloc(&tl.tmem_base, 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tl.tmem_base;
+    SeqView sv;
+    sv.pack = t_pack; sv.tiles = t_tiles; sv.len = t_len; sv.start = t_start;
 
     // ranges over min(grid, items) CTAs, so that every CTA that has a range has a non-empty one
-    const int items = tl.seq.tiles[a.p.num_seqs] * a.p.num_kv_heads;
+    const int items = t_tiles[B] * a.p.num_kv_heads;
     const int ctas = max(1, min((int)gridDim.x, items));
     const bool active = (int)blockIdx.x < ctas;
     const int item0 = active ? range_begin(blockIdx.x, items, ctas) : 0;
@@ -763,26 +905,27 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     // PASS 1 or 2: that pass alone; PASS 3: both passes in this launch (all CTAs co-resident)
     if (warp < kEpiWarps) {
         EpiState es;
-        if (PASS != 2) epilogue_pass1(a, tl, tmem_base, item0, item1, es);
+        if (PASS != 2) epilogue_pass1(a, tl, tmem_base, item1 - item0, es);
         if (PASS == 3) {
             // publish: this CTA's partials are in memory
             __threadfence();
             epi_sync(tl, es.ephase);
             if (threadIdx.x == 0)
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(a.epoch) : "memory");
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(1u) : "memory");
         }
-        if (PASS != 1) epilogue_pass2(a, tl, tmem_base, item0, item1, items, ctas, es);
+        if (PASS != 1) epilogue_pass2(a, tl, sv, tmem_base, item1 - item0, items, ctas, es);
     } else if (warp == kEpiWarps) {
         if (lane == 0) {
             RingState rs;
-            if (PASS != 2) producer_loop<1>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1, rs);
-            if (PASS != 1) producer_loop<2>(a, &mapq, &mapk, smem_q, smem_k, tl, item0, item1, rs);
+            if (PASS != 2) producer_loop(a, &mapq, &mapk, smem_q, smem_k, tl, sv, item0, item1, rs);
+            if (PASS != 1) producer_loop(a, &mapq, &mapk, smem_q, smem_k, tl, sv, item0, item1, rs);
         }
     } else {
         if (lane == 0) {
             MmaState ms;
-            if (PASS != 2) mma_loop<1>(a, smem_q, smem_k, tl, tmem_base, item0, item1, ms);
-            if (PASS != 1) mma_loop<2>(a, smem_q, smem_k, tl, tmem_base, item0, item1, ms);
+            if (PASS != 2) mma_loop_pass1(a, smem_q, smem_k, tl, tmem_base, item1 - item0, ms);
+            if (PASS == 3) drain_pass1(tl, ms);
+            if (PASS != 1 && !tl.abort_flag) mma_loop_pass2(a, smem_q, smem_k, tl, tmem_base, item1 - item0, ms);
         }
     }
     __syncwarp();
@@ -821,19 +964,53 @@ bool shape_for(const refree_params &p, TcShape &sh)
     const int64_t R = (int64_t)G * p.window;
     if (R < 32 || R > kMaxRowsTc) return false;
     sh.R = (int)R;
-    sh.cblocks = (sh.R + kTile - 1) / kTile;
-    if (sh.R % (16 * sh.cblocks) != 0) return false;      // accumulators are read in chunks of 16 columns
-    sh.ncol = sh.R / sh.cblocks;
     sh.rblocks = (sh.R + kTile - 1) / kTile;
     sh.Rpad = sh.rblocks * kTile;
+    sh.cblocks = sh.R > 256 ? 2 : 1;
+    sh.ncol = ((sh.R + sh.cblocks - 1) / sh.cblocks + 15) / 16 * 16;   // rows past R are masked by L = +inf
     sh.stages = sh.Rpad <= 256 ? 4 : 2;
     sh.rank4 = p.k_stride_seq != 0;
     return true;
 }
 
-size_t smem_bytes(const TcShape &sh)
+size_t smem_bytes(const TcShape &sh, int num_seqs)
 {
-    return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + sizeof(TcSmemTail);
+    return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + sizeof(TcSmemTail) +
+           (size_t)(4 * num_seqs + 2) * sizeof(int32_t);
+}
+
+constexpr size_t kSmemLimit = 232448;
+
+// Per-device facts, looked up once per device under a lock.
+struct DevInfo { bool ready = false; int sms = 0; bool coop = false; cudaError_t err = cudaSuccess; };
+std::mutex g_dev_mutex;
+DevInfo g_dev[64];
+
+cudaError_t device_info(DevInfo &out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    DevInfo &d = g_dev[dev];
+    if (!d.ready) {
+        int n = 0, coop = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) coop = 0;
+        d.sms = std::min(n, kMaxCtas);
+        d.coop = coop != 0;
+        d.ready = true;
+    }
+    out = d;
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -843,6 +1020,7 @@ bool score_tc_supported(const refree_params &p)
     TcShape sh;
     if (!shape_for(p, sh)) return false;
     if (p.kv_tokens <= 0 || p.kv_tokens > 0x7fffffffLL) return false;
+    if (smem_bytes(sh, p.num_seqs) > kSmemLimit) return false;
     return encode_fn() != nullptr;
 }
 
@@ -875,29 +1053,11 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
-    static int sm_count[64] = {};
-    static bool coop_ok[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DevInfo di;
+    cudaError_t e = device_info(di);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (sm_count[dev] == 0) {
-        int n = 0;
-        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(score_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-        if (e != cudaSuccess) return e;
-        int coop = 0;
-        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) coop = 0;
-        coop_ok[dev] = coop != 0;
-        sm_count[dev] = std::min(n, kMaxCtas);
-    }
     const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
-    const int ctas = (int)std::max<int64_t>(1, std::min<int64_t>(sm_count[dev], max_items));
+    const int ctas = (int)std::max<int64_t>(1, std::min<int64_t>(di.sms, max_items));
     TcArgs a;
     a.p = p;
     a.sh = sh;
@@ -908,19 +1068,15 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.scores = scores;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;
-    const size_t smem = smem_bytes(sh);
-    if (smem > 232448) return cudaErrorInvalidValue;
+    const size_t smem = smem_bytes(sh, p.num_seqs);
+    if (smem > kSmemLimit) return cudaErrorInvalidValue;
     a.flags = nullptr;
-    a.epoch = 0;
-    if (coop_ok[dev]) {
+    if (di.coop) {
         // Both passes in one cooperative launch (co-residency of all CTAs is what makes the wait of pass 2
-        // on other CTAs' pass 1 safe).  The flags hold a per-call token, so a workspace left over from an
-        // earlier call needs no clearing.
-        static std::atomic<uint32_t> token{0x5eed1234u};
-        uint32_t epoch = token.fetch_add(1u, std::memory_order_relaxed) + 1u;
-        if (epoch == 0u) epoch = token.fetch_add(1u, std::memory_order_relaxed) + 1u;
+        // on other CTAs' pass 1 safe).  The flags are cleared on the stream before the launch.
         a.flags = reinterpret_cast<uint32_t *>(ws + lay.cnt_off);
-        a.epoch = epoch;
+        e = cudaMemsetAsync(a.flags, 0, (size_t)kMaxCtas * sizeof(uint32_t), st);
+        if (e != cudaSuccess) return e;
         void *args[3] = {(void *)&mapq, (void *)&mapk, (void *)&a};
         const cudaError_t ce = cudaLaunchCooperativeKernel((const void *)score_tc_kernel<3>, dim3(ctas), dim3(kThreadsTc),
                                                            args, smem, st);

@@ -176,6 +176,17 @@ def test_select_matches_masked_norm_definition(rank_mode, scope, T):
             u = s * Hkv + g
             kept = sel.kept_idx[sel.offsets[u]:sel.offsets[u + 1]]
             np.testing.assert_array_equal(kept, np.sort(order[:max(j, 1)]))
+            # the criterion curve sqrt(C_j / C_n) of Eq. 3 and the distance of the decision from a tie: the
+            # parity rules excuse a budget mismatch only through these two, so they are pinned like the rest
+            curve = np.sqrt(np.cumsum(sq[order]) / sq.sum())
+            np.testing.assert_allclose(sel.ratio[g, off:off + n], curve, rtol=1e-13, atol=0)
+            crossed = (1.0 - curve < Tf).any()
+            if crossed:
+                near = [abs(curve[j - 1] - (1.0 - Tf))] + ([abs(curve[j - 2] - (1.0 - Tf))] if j > 1 else [])
+                want_gap = min(near)
+            else:
+                want_gap = abs(1.0 - (1.0 - Tf))
+            np.testing.assert_allclose(sel.gap[s, g], want_gap, rtol=1e-9, atol=1e-15)
         off += n
     np.testing.assert_array_equal(sel.offsets, np.concatenate([[0], np.cumsum(sel.lengths.reshape(-1))]))
 

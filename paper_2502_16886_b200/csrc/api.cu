@@ -469,6 +469,57 @@ refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
     if (!workspace || workspace_bytes < 2 * lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
         return REFREE_ERR_WORKSPACE;
     if (num_layers == 0) return REFREE_OK;
+    // Position ranking on the tensor-core path with rows of a unit contiguous: one stream, the scoring kernel
+    // of layer l moves the kept rows of layer l - 1 with a warp of its own, the last layer is compacted by a
+    // launch of its own.  No internal streams or events.
+    bool fused = num_layers >= 2 && total_tokens > 0 && !p->force_full && p->rank_mode == REFREE_RANK_POSITION &&
+                 score_tc_can_copy(*p, total_tokens);
+    for (int l = 0; l < num_layers && fused; ++l) fused = use_tc(*p, q_win[l]);
+    if (fused) {
+        // launch j (0 <= j <= L): column pass and stopping rule of layer j - 1, row pass of layer j, rows of
+        // layer j - 2; then the last two layers' rows
+        cudaStream_t cs = (cudaStream_t)stream;
+        auto layer_of = [&](int l) {
+            TcLayer t;
+            char *ws = (char *)workspace + (size_t)(l & 1) * lay.total;
+            t.q_win = q_win[l];
+            t.k = k[l];
+            t.ws = ws;
+            t.scores = reinterpret_cast<float *>(ws + lay.scores_off);
+            t.groups = p->scope == REFREE_SCOPE_HEAD ? reinterpret_cast<GroupPartial *>(ws + lay.grp_off) : nullptr;
+            return t;
+        };
+        auto job_of = [&](int l) {
+            TcCopyJob job;
+            job.k = (const unsigned char *)k[l];
+            job.v = (const unsigned char *)v[l];
+            job.k_out = (unsigned char *)k_out[l];
+            job.v_out = (unsigned char *)v_out[l];
+            job.lengths = lengths[l];
+            job.offsets_out = offsets[l];
+            job.capacity_rows = capacity_rows;
+            job.nslots = 0;
+            return job;
+        };
+        for (int j = 0; j <= num_layers; ++j) {
+            TcLayer beg, fin;
+            TcCopyJob job;
+            if (j < num_layers) beg = layer_of(j);
+            if (j >= 1) fin = layer_of(j - 1);
+            if (j >= 2) job = job_of(j - 2);
+            if (launch_score_tc_pipe(*p, j < num_layers ? &beg : nullptr, j >= 1 ? &fin : nullptr, seq_start, seq_len,
+                                     total_tokens, lay, device_status, cs, j >= 2 ? &job : nullptr) != cudaSuccess)
+                return REFREE_ERR_CUDA;
+            if (j >= 1 &&
+                launch_select(*p, fin.scores, seq_len, total_tokens, lengths[j - 1], offsets[j - 1], nullptr, capacity_rows,
+                              fin.ws, lay, device_status, cs, false, fin.groups) != cudaSuccess)
+                return REFREE_ERR_CUDA;
+        }
+        // the rows of the last layer; those of the one before it went with the last scoring launch
+        const int l = num_layers - 1;
+        return from_cuda(launch_compact(*p, k[l], v[l], seq_start, seq_len, lengths[l], offsets[l], nullptr, true,
+                                        offsets[l], k_out[l], v_out[l], capacity_rows, device_status, cs));
+    }
     LayerPipe *lp = layer_pipe();
     if (!lp) return REFREE_ERR_CUDA;
     cudaStream_t cs = (cudaStream_t)stream;

@@ -124,12 +124,42 @@ cudaError_t launch_score_generic(const refree_params &p, const void *q_win, cons
                                  int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
                                  int32_t *dev_status, cudaStream_t st);
 
+// Rows of another layer (position ranking: a prefix and a suffix per unit) that the tensor-core scoring
+// kernel moves with a warp of its own while it scores, HBM being nearly idle then.  The budgets are read
+// on the device; the kernel forms their running sum itself.
+struct TcCopyJob {
+    const unsigned char *k, *v;     // source cache (same strides and sequences as the scored layer)
+    unsigned char *k_out, *v_out;   // dense outputs [capacity_rows, d]
+    const int32_t *lengths;         // [num_seqs * num_kv_heads] budgets
+    int64_t *offsets_out;           // nullable: [units + 1] running sum of the budgets
+    int64_t capacity_rows;
+    int nslots;                     // pieces in flight (0: nothing to move); set by the launcher
+};
+
 // Returns false when the shape is outside what the tensor-core path handles.
 bool score_tc_supported(const refree_params &p);
+// True when launch_score_tc can also carry a TcCopyJob for these parameters (rows of a unit contiguous in
+// K and V, few enough units, shared memory left for the pieces in flight).
+bool score_tc_can_copy(const refree_params &p, int64_t total_tokens);
+// Both passes of one layer in one cooperative launch (two plain launches where that is not available).
 cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
                             const int32_t *seq_start, const int32_t *seq_len,
                             int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
                             int32_t *dev_status, cudaStream_t st, GroupPartial *groups = nullptr);
+
+// One layer of a run of layers, as the scoring launches of the run see it.
+struct TcLayer {
+    const void *q_win, *k;
+    float *scores;          // [Hkv, total_tokens]
+    char *ws;               // the layer's workspace (partials between its two passes)
+    GroupPartial *groups;   // nullable
+};
+// One launch of a run: the column pass of `finish`, then the row pass of `begin` (either may be null), and the
+// rows of `copy` (nullable) moved beside them.
+cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, const TcLayer *finish,
+                                 const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                                 const Workspace &lay, int32_t *dev_status, cudaStream_t st,
+                                 const TcCopyJob *copy = nullptr);
 
 // Single query row per head (the paper's default reduced attention): a stream over K on the fp32 pipes.
 bool score_w1_supported(const refree_params &p);

@@ -42,8 +42,12 @@ namespace refree {
 namespace {
 
 constexpr int kEpiWarps = 16;
-constexpr int kThreadsTc = (kEpiWarps + 2) * 32;
+constexpr int kThreadsTc = (kEpiWarps + 3) * 32;    // + TMA warp, MMA warp, copy warp
+constexpr int kMaxCopySlots = 6;
+constexpr int kMaxCopyUnits = 1024;                 // units whose running budget sum fits the CTA's table
 constexpr int kD = 128;
+constexpr int kCopyRows = 32;                       // rows of one piece of the in-kernel row copy
+constexpr int kCopySlot = kCopyRows * kD * 2;       // 8 KB
 constexpr int kHalfBytes = kTile * 128;          // one 64-column half of a 128-row tile: 16 KB
 constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr int kMaxRowsTc = 512;
@@ -218,6 +222,7 @@ struct TcSmemTail {
     uint64_t acc_full[4], acc_empty[4];       // pass 1: accumulator (pair * 2 + slot), 128 tensor-memory columns each
     uint64_t p2_full[2], p2_empty[2];         // pass 2: accumulators of 256 columns
     uint64_t chunk_ready[4];                  // pass 2: the other column chunks have staged their shares of a tile
+    uint64_t c_full[kMaxCopySlots];           // row copy: a piece has landed in its slot
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) ItemInfo info[kInfoRing];
@@ -287,12 +292,16 @@ struct TcArgs {
     refree_params p;
     TcShape sh;
     const int32_t *seq_start, *seq_len;
-    float2 *part;        // [2 (ctas + units)][Rpad]: one record per (CTA, unit, column half)
+    // Pass 1 writes the partials of layer `la`, pass 2 reads those of layer `lb` and writes its scores (the same
+    // layer when both passes of one layer run in a launch; consecutive layers of a run otherwise).
+    float2 *part_a;      // [2 (ctas + units)][Rpad]: one record per (CTA, unit, column half)
+    const float2 *part_b;
     GroupPartial *groups; // nullable: per 32 positions, exact sum of squared scores for the stopping rule
-    uint32_t *flags;     // fused launch: flags[c] != 0 once CTA c has written its pass-1 partials (zeroed before the launch)
     float *scores;
+    uint32_t *flags;     // one layer per launch: flags[c] != 0 once CTA c has written its pass-1 partials (zeroed before the launch)
     int64_t total_tokens;
     int32_t *dev_status;
+    TcCopyJob cj;          // rows of an earlier layer to move while this layer is scored (nslots == 0: none)
 };
 
 // Barrier among the epilogue warps, built on an mbarrier so that it is bounded like
@@ -433,6 +442,18 @@ __device__ inline bool drain_pass1(TcSmemTail &tl, const MmaState &ms)
     return ok;
 }
 
+// The other way round (a launch that finishes one layer and then begins the next).
+__device__ inline bool drain_pass2(TcSmemTail &tl, const MmaState &ms)
+{
+    bool ok = true;
+    for (int buf = 0; buf < 2 && ok; ++buf) {
+        const uint32_t uses = (ms.cnt2 + (buf ? 0u : 1u)) >> 1;
+        if (uses) ok = mbar_wait(&tl.p2_empty[buf], (uses - 1u) & 1u, &tl.abort_flag);
+    }
+    if (ok) tc_fence_after();
+    return ok;
+}
+
 // Pass 2: D[position, row] = K_tile Q^T, `ncol` rows of Q per product.
 __device__ inline void mma_loop_pass2(const TcArgs &a, unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl,
                                       uint32_t tmem_base, int nitems, MmaState &ms)
@@ -540,7 +561,7 @@ __device__ inline void epilogue_pass1(const TcArgs &a, TcSmemTail &tl, uint32_t 
             const int rb = pair + 2 * j;
             const int row = rb * kTile + lane_base + lane;
             if (rb < sh.rblocks && row < sh.R)
-                a.part[((int64_t)(blockIdx.x + u) * 2 + half) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
+                a.part_a[((int64_t)(blockIdx.x + u) * 2 + half) * sh.Rpad + row] = make_float2(cref[j], zsum[j]);
             cref[j] = -INFINITY;
             zsum[j] = 0.f;
         }
@@ -784,7 +805,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
 #pragma unroll
                             for (int q = 0; q < 8; ++q)
                                 pr[q] = (s0 + q * per_row <= s_hi)
-                                            ? __ldcg(&a.part[(int64_t)(s0 + q * per_row) * sh.Rpad + r])
+                                            ? __ldcg(&a.part_b[(int64_t)(s0 + q * per_row) * sh.Rpad + r])
                                             : make_float2(-INFINITY, 0.f);
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
@@ -842,25 +863,153 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
     if (chunk == 0 && ok) finish_pending();
 }
 
-// ---------------------------------------------------------------- kernels ----
-template <int PASS>
-__global__ void __launch_bounds__(kThreadsTc, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant__ CUtensorMap mapk, TcArgs a)
+// ------------------------------------------------------------- row copy -----
+// Compaction of another layer by one warp of the scoring CTA (position ranking: the kept rows of a unit
+// are rows [0, head) and [n - (b - head), n) of its cache, contiguous in memory when a unit's rows are).
+// Destination rows are cut into pieces of 32 rows; piece k belongs to CTA k mod grid, and inside the CTA
+// to one lane of the warp, which owns a slot of shared memory.  A piece travels global -> shared -> global
+// with the bulk-copy engine (no tensor map, no multicast): the load is signalled on the slot's mbarrier,
+// the store is a bulk group.  Nothing here touches the registers or pipes of the scoring warps.
+__device__ inline void copy_loop(const TcArgs &a, TcSmemTail &tl, const SeqView &sv, unsigned char *smem_c, int32_t *coff)
 {
+    const TcCopyJob &cj = a.cj;
+    const int lane = threadIdx.x & 31;
+    const int Hkv = a.p.num_kv_heads, U = a.p.num_seqs * Hkv;
+    // running sum of the budgets (clamped to [0, n]); a budget out of range is reported
+    int carry = 0;
+    bool bad = false;
+    for (int base = 0; base < U; base += 32) {
+        const int u = base + lane;
+        int b = 0;
+        if (u < U) {
+            b = cj.lengths[u];
+            const int n = sv.len[u / Hkv];
+            if (b < 0 || b > n) { bad = true; b = max(0, min(b, n)); }
+        }
+        int x = b;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (u < U) coff[u] = carry + x - b;
+        carry += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) coff[U] = carry;
+    __syncwarp();
+    bad = __any_sync(0xffffffffu, bad);
+    const int64_t rows = min((int64_t)carry, cj.capacity_rows);
+    if (blockIdx.x == 0) {
+        if (cj.offsets_out)
+            for (int u = lane; u <= U; u += 32) cj.offsets_out[u] = coff[u];
+        if (lane == 0 && (bad || (int64_t)carry > cj.capacity_rows) && a.dev_status)
+            atomicOr(a.dev_status, REFREE_DEV_CAPACITY);
+    }
+    const int nslots = cj.nslots;
+    if (lane >= nslots || rows <= 0) return;
+
+    // Lane j owns slot j and every nslots-th piece of this CTA; the lanes move in step: all load, all wait,
+    // all store, all wait until their stores have read the slots.
+    const unsigned workers = (1u << nslots) - 1u;
+    const int64_t k_tok = a.p.k_stride_tok * 2, v_tok = a.p.v_stride_tok * 2;      // bytes (bf16)
+    const int64_t pieces_per_array = (rows + kCopyRows - 1) / kCopyRows, pieces = 2 * pieces_per_array;
+    int64_t next = blockIdx.x + (int64_t)lane * gridDim.x;      // next piece of this lane
+    const int64_t step = (int64_t)nslots * gridDim.x;
+    int r_cur = 0, r_end = 0, u_cur = 0, arr = 0;      // rows [r_cur, r_end) of the current piece still to cut
+    unsigned char *slot = smem_c + (size_t)lane * kCopySlot;
+    uint64_t *bar = &tl.c_full[lane];
+    // the moved rows are used once: they should not push the scored layer's K tiles out of L2
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    uint32_t loads = 0;
+    bool ok = true;
+    while (ok) {
+        // the next run of rows that is contiguous in source and destination
+        bool has = true;
+        if (r_cur >= r_end) {
+            if (next >= pieces) {
+                has = false;
+            } else {
+                arr = next >= pieces_per_array ? 1 : 0;
+                const int64_t pk = next - (arr ? pieces_per_array : 0);
+                next += step;
+                r_cur = (int)(pk * kCopyRows);
+                r_end = (int)min((int64_t)r_cur + kCopyRows, rows);
+                int lo = 0, hi = U;                             // largest u with coff[u] <= r_cur
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (coff[mid] <= r_cur) lo = mid; else hi = mid;
+                }
+                u_cur = lo;
+            }
+        }
+        if (!__any_sync(workers, has)) break;
+        unsigned char *dst = nullptr;
+        uint32_t bytes = 0;
+        if (has) {
+            while (coff[u_cur + 1] <= r_cur) ++u_cur;           // skip units that keep nothing (r_cur < rows <= coff[U])
+            const int b = coff[u_cur + 1] - coff[u_cur], t = r_cur - coff[u_cur];
+            const int sq = u_cur / Hkv, g = u_cur - sq * Hkv;
+            const int n = sv.len[sq], head = min(b, min(a.p.sink, n));
+            int src_row, run;
+            if (t < head) { src_row = t; run = head - t; }
+            else { src_row = n - b + t; run = b - t; }
+            run = min(run, r_end - r_cur);
+            const int64_t tok = (int64_t)sv.start[sq] + src_row;
+            const unsigned char *src =
+                arr == 0 ? cj.k + ((int64_t)sq * a.p.k_stride_seq + (int64_t)g * a.p.k_stride_head) * 2 + tok * k_tok
+                         : cj.v + ((int64_t)sq * a.p.v_stride_seq + (int64_t)g * a.p.v_stride_head) * 2 + tok * v_tok;
+            dst = (arr ? cj.v_out : cj.k_out) + (int64_t)r_cur * (kD * 2);
+            bytes = (uint32_t)run * (kD * 2);
+            r_cur += run;
+            mbar_expect_tx(bar, bytes);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                         ::"r"(smem_u32(slot)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+            ok = mbar_wait(bar, loads & 1u, &tl.abort_flag);
+            ++loads;
+            if (ok) {
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                             ::"l"(dst), "r"(smem_u32(slot)), "r"(bytes), "l"(pol) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
+        }
+        ok = !__any_sync(workers, !ok) && !tl.abort_flag;
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// ---------------------------------------------------------------- kernels ----
+// MODE 1: pass 1 alone; 2: pass 2 alone; 3: both passes of one layer (cooperative launch: pass 2 waits for the
+// pass-1 flags of other CTAs); 4: pass 2 of one layer (maps `_b`), then pass 1 of the next (maps `_a`) - the
+// steady state of a run of layers, where the partials pass 2 reads were completed by the launch before.
+template <int MODE>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constant__ CUtensorMap mapk_a,
+                const __grid_constant__ CUtensorMap mapq_b, const __grid_constant__ CUtensorMap mapk_b, TcArgs a)
+{
+    constexpr bool P1 = MODE != 2, P2 = MODE != 1;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const TcShape &sh = a.sh;
     unsigned char *smem_q = smem;
     unsigned char *smem_k = smem + (size_t)sh.Rpad * 256;
-    TcSmemTail &tl = *reinterpret_cast<TcSmemTail *>(smem_k + (size_t)sh.stages * kTileBytes);
+    unsigned char *smem_c = smem_k + (size_t)sh.stages * kTileBytes;        // pieces of the row copy
+    TcSmemTail &tl = *reinterpret_cast<TcSmemTail *>(smem_c + (size_t)a.cj.nslots * kCopySlot);
     int32_t *tab = reinterpret_cast<int32_t *>(&tl + 1);
     const int B = a.p.num_seqs;
     int32_t *t_pack = tab, *t_tiles = tab + (B + 1), *t_len = tab + 2 * (B + 1), *t_start = tab + 2 * (B + 1) + B;
+    int32_t *coff = tab + 4 * B + 2;             // row copy: running sum of the budgets, units + 1 entries
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == kEpiWarps * 32) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapq) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapk) : "memory");
+        if (P1) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapq_a) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapk_a) : "memory");
+        }
+        if (P2) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapq_b) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&mapk_b) : "memory");
+        }
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) { mbar_init(&tl.k_full[s], 1); mbar_init(&tl.k_empty[s], 1); }
@@ -870,6 +1019,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
         for (int b = 0; b < 2; ++b) { mbar_init(&tl.p2_full[b], 1); mbar_init(&tl.p2_empty[b], kEpiWarps); }
         for (int b = 0; b < 4; ++b) mbar_init(&tl.chunk_ready[b], 12);      // the twelve warps of chunks 1..3
         mbar_init(&tl.epi_bar, kEpiWarps);
+        for (int b = 0; b < kMaxCopySlots; ++b) mbar_init(&tl.c_full[b], 1);
         tl.abort_flag = 0;
         fence_barrier_init();
     }
@@ -902,30 +1052,38 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq, const __grid_constant_
     const int item0 = active ? range_begin(blockIdx.x, items, ctas) : 0;
     const int item1 = active ? range_begin(blockIdx.x + 1, items, ctas) : 0;
 
-    // PASS 1 or 2: that pass alone; PASS 3: both passes in this launch (all CTAs co-resident)
+    const int nitems = item1 - item0;
     if (warp < kEpiWarps) {
         EpiState es;
-        if (PASS != 2) epilogue_pass1(a, tl, tmem_base, item1 - item0, es);
-        if (PASS == 3) {
+        if (MODE == 4) epilogue_pass2(a, tl, sv, tmem_base, nitems, items, ctas, es);
+        if (P1) epilogue_pass1(a, tl, tmem_base, nitems, es);
+        if (MODE == 3) {
             // publish: this CTA's partials are in memory
             __threadfence();
             epi_sync(tl, es.ephase);
             if (threadIdx.x == 0)
                 asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(1u) : "memory");
         }
-        if (PASS != 1) epilogue_pass2(a, tl, sv, tmem_base, item1 - item0, items, ctas, es);
+        if (P2 && MODE != 4) epilogue_pass2(a, tl, sv, tmem_base, nitems, items, ctas, es);
     } else if (warp == kEpiWarps) {
         if (lane == 0) {
             RingState rs;
-            if (PASS != 2) producer_loop(a, &mapq, &mapk, smem_q, smem_k, tl, sv, item0, item1, rs);
-            if (PASS != 1) producer_loop(a, &mapq, &mapk, smem_q, smem_k, tl, sv, item0, item1, rs);
+            if (MODE == 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs);
+            if (P1) producer_loop(a, &mapq_a, &mapk_a, smem_q, smem_k, tl, sv, item0, item1, rs);
+            if (P2 && MODE != 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs);
         }
+    } else if (warp == kEpiWarps + 2) {
+        if (a.cj.nslots > 0) copy_loop(a, tl, sv, smem_c, coff);
     } else {
         if (lane == 0) {
             MmaState ms;
-            if (PASS != 2) mma_loop_pass1(a, smem_q, smem_k, tl, tmem_base, item1 - item0, ms);
-            if (PASS == 3) drain_pass1(tl, ms);
-            if (PASS != 1 && !tl.abort_flag) mma_loop_pass2(a, smem_q, smem_k, tl, tmem_base, item1 - item0, ms);
+            if (MODE == 4) {
+                mma_loop_pass2(a, smem_q, smem_k, tl, tmem_base, nitems, ms);
+                drain_pass2(tl, ms);
+            }
+            if (P1 && !tl.abort_flag) mma_loop_pass1(a, smem_q, smem_k, tl, tmem_base, nitems, ms);
+            if (MODE == 3) drain_pass1(tl, ms);
+            if (P2 && MODE != 4 && !tl.abort_flag) mma_loop_pass2(a, smem_q, smem_k, tl, tmem_base, nitems, ms);
         }
     }
     __syncwarp();
@@ -973,10 +1131,11 @@ bool shape_for(const refree_params &p, TcShape &sh)
     return true;
 }
 
-size_t smem_bytes(const TcShape &sh, int num_seqs)
+size_t smem_bytes(const TcShape &sh, int num_seqs, int copy_slots = 0, int copy_units = 0)
 {
-    return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + sizeof(TcSmemTail) +
-           (size_t)(4 * num_seqs + 2) * sizeof(int32_t);
+    return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + (size_t)copy_slots * kCopySlot +
+           sizeof(TcSmemTail) + (size_t)(4 * num_seqs + 2) * sizeof(int32_t) +
+           (copy_slots ? (size_t)(copy_units + 1) * sizeof(int32_t) : 0);
 }
 
 constexpr size_t kSmemLimit = 232448;
@@ -1004,6 +1163,8 @@ cudaError_t device_info(DevInfo &out)
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(score_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(score_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+        if (e != cudaSuccess) return e;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) coop = 0;
         d.sms = std::min(n, kMaxCtas);
         d.coop = coop != 0;
@@ -1013,7 +1174,30 @@ cudaError_t device_info(DevInfo &out)
     return cudaSuccess;
 }
 
+// Ring depth and pieces in flight when the launch also copies rows: the K ring gives up a stage where it
+// has four, and the pieces take what is left.  False when fewer than three pieces would fit.
+bool copy_shape(const refree_params &p, TcShape &sh, int &nslots)
+{
+    const int U = p.num_seqs * p.num_kv_heads;
+    if (sh.stages > 3) sh.stages = 3;
+    for (nslots = kMaxCopySlots; nslots >= 3; --nslots)
+        if (smem_bytes(sh, p.num_seqs, nslots, U) <= kSmemLimit) return true;
+    return false;
+}
+
 }  // namespace
+
+bool score_tc_can_copy(const refree_params &p, int64_t total_tokens)
+{
+    TcShape sh;
+    int nslots = 0;
+    if (!shape_for(p, sh)) return false;
+    if (p.k_stride_tok != kD || p.v_stride_tok != kD) return false;          // a unit's rows back to back
+    if ((int64_t)p.num_seqs * p.num_kv_heads > kMaxCopyUnits) return false;
+    if ((int64_t)p.num_kv_heads * total_tokens > 0x7fffffffLL) return false;  // row counts held in 32 bits
+    if (p.rank_mode != REFREE_RANK_POSITION && !p.force_full) return false;
+    return copy_shape(p, sh, nslots);
+}
 
 bool score_tc_supported(const refree_params &p)
 {
@@ -1024,16 +1208,13 @@ bool score_tc_supported(const refree_params &p)
     return encode_fn() != nullptr;
 }
 
-cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
-                            const int32_t *seq_start, const int32_t *seq_len,
-                            int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
-                            int32_t *dev_status, cudaStream_t st, GroupPartial *groups)
+namespace {
+
+cudaError_t encode_maps(const refree_params &p, const TcShape &sh, const void *q_win, const void *k, CUtensorMap &mapq,
+                        CUtensorMap &mapk)
 {
-    TcShape sh;
-    if (!shape_for(p, sh)) return cudaErrorInvalidValue;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
-    CUtensorMap mapq, mapk;
     {
         const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_seqs * p.num_q_heads * p.window};
         const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
@@ -1053,8 +1234,24 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
+    return cudaSuccess;
+}
+
+}  // namespace
+
+// Both passes of one layer.
+cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const void *k,
+                            const int32_t *seq_start, const int32_t *seq_len,
+                            int64_t total_tokens, float *scores, char *ws, const Workspace &lay,
+                            int32_t *dev_status, cudaStream_t st, GroupPartial *groups)
+{
+    TcShape sh;
+    if (!shape_for(p, sh)) return cudaErrorInvalidValue;
+    CUtensorMap mapq, mapk;
+    cudaError_t e = encode_maps(p, sh, q_win, k, mapq, mapk);
+    if (e != cudaSuccess) return e;
     DevInfo di;
-    cudaError_t e = device_info(di);
+    e = device_info(di);
     if (e != cudaSuccess) return e;
     const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
     const int ctas = (int)std::max<int64_t>(1, std::min<int64_t>(di.sms, max_items));
@@ -1063,11 +1260,13 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.sh = sh;
     a.seq_start = seq_start;
     a.seq_len = seq_len;
-    a.part = reinterpret_cast<float2 *>(ws + lay.part_off);
+    a.part_a = reinterpret_cast<float2 *>(ws + lay.part_off);
+    a.part_b = a.part_a;
     a.groups = groups;
     a.scores = scores;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;
+    a.cj = TcCopyJob{};
     const size_t smem = smem_bytes(sh, p.num_seqs);
     if (smem > kSmemLimit) return cudaErrorInvalidValue;
     a.flags = nullptr;
@@ -1077,7 +1276,7 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
         a.flags = reinterpret_cast<uint32_t *>(ws + lay.cnt_off);
         e = cudaMemsetAsync(a.flags, 0, (size_t)kMaxCtas * sizeof(uint32_t), st);
         if (e != cudaSuccess) return e;
-        void *args[3] = {(void *)&mapq, (void *)&mapk, (void *)&a};
+        void *args[5] = {(void *)&mapq, (void *)&mapk, (void *)&mapq, (void *)&mapk, (void *)&a};
         const cudaError_t ce = cudaLaunchCooperativeKernel((const void *)score_tc_kernel<3>, dim3(ctas), dim3(kThreadsTc),
                                                            args, smem, st);
         if (ce == cudaSuccess) {
@@ -1087,9 +1286,56 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
         (void)cudaGetLastError();        // not launchable as one grid here: fall back to one launch per pass
         a.flags = nullptr;
     }
-    score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
-    score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, a);
+    score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, mapq, mapk, a);
+    score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq, mapk, mapq, mapk, a);
     count_launches(2);
+    return cudaGetLastError();
+}
+
+// One launch of a run of layers: pass 2 of `finish` (nullable), then pass 1 of `begin` (nullable), and the rows
+// of `copy` (nullable) beside them.  The partials that pass 2 reads were completed by an earlier launch on the
+// stream, so no CTA waits for another and the launch is an ordinary one.
+cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, const TcLayer *finish,
+                                 const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
+                                 const Workspace &lay, int32_t *dev_status, cudaStream_t st, const TcCopyJob *copy)
+{
+    if (!begin && !finish) return cudaErrorInvalidValue;
+    TcShape sh;
+    if (!shape_for(p, sh)) return cudaErrorInvalidValue;
+    int copy_slots = 0;
+    if (copy && !copy_shape(p, sh, copy_slots)) return cudaErrorInvalidValue;
+    CUtensorMap mapq_a, mapk_a, mapq_b, mapk_b;
+    cudaError_t e = cudaSuccess;
+    if (begin && (e = encode_maps(p, sh, begin->q_win, begin->k, mapq_a, mapk_a)) != cudaSuccess) return e;
+    if (finish && (e = encode_maps(p, sh, finish->q_win, finish->k, mapq_b, mapk_b)) != cudaSuccess) return e;
+    if (!begin) { mapq_a = mapq_b; mapk_a = mapk_b; }
+    if (!finish) { mapq_b = mapq_a; mapk_b = mapk_a; }
+    DevInfo di;
+    e = device_info(di);
+    if (e != cudaSuccess) return e;
+    const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
+    // with rows to move, every SM takes part whatever the number of scoring items
+    const int ctas = copy ? di.sms : (int)std::max<int64_t>(1, std::min<int64_t>(di.sms, max_items));
+    TcArgs a;
+    a.p = p;
+    a.sh = sh;
+    a.seq_start = seq_start;
+    a.seq_len = seq_len;
+    a.part_a = begin ? reinterpret_cast<float2 *>(begin->ws + lay.part_off) : nullptr;
+    a.part_b = finish ? reinterpret_cast<const float2 *>(finish->ws + lay.part_off) : nullptr;
+    a.groups = finish ? finish->groups : nullptr;
+    a.scores = finish ? finish->scores : nullptr;
+    a.flags = nullptr;
+    a.total_tokens = total_tokens;
+    a.dev_status = dev_status;
+    if (copy) a.cj = *copy; else a.cj = TcCopyJob{};
+    a.cj.nslots = copy ? copy_slots : 0;
+    const size_t smem = smem_bytes(sh, p.num_seqs, a.cj.nslots, p.num_seqs * p.num_kv_heads);
+    if (smem > kSmemLimit) return cudaErrorInvalidValue;
+    if (begin && finish) score_tc_kernel<4><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
+    else if (begin) score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
+    else score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
+    count_launches(1);
     return cudaGetLastError();
 }
 

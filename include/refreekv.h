@@ -14,9 +14,18 @@
  *
  * Conventions common to every entry point
  *   - All array arguments are DEVICE pointers owned by the caller unless the
- *     function name ends in `_host`.  The library allocates nothing, never
- *     synchronises the device (except the `_host` variant), and enqueues all
+ *     function name ends in `_host`.  The library allocates no device memory
+ *     and never synchronises the device (except the `_host` variants, which
+ *     also create and destroy streams and events per call), and enqueues its
  *     work on the caller's stream (`stream` is a cudaStream_t passed as void*).
+ *     refree_compress_layers may, for shapes outside its one-stream path, use
+ *     two internal streams and a few events that are made once per device and
+ *     kept until the process exits; they fork from and join the caller's stream.
+ *   - The first call of an entry point on a device sets kernel attributes and
+ *     reads device properties; make it outside any stream capture.
+ *   - Limits, all reported as REFREE_ERR_UNSUPPORTED: num_seqs <= 1024;
+ *     num_seqs * num_kv_heads <= 65535; (num_q_heads / num_kv_heads) * window
+ *     <= 1024; head_dim 64 or 128; 16-byte aligned K/V base pointers and strides.
  *   - Element (s, g, i, :) of K lives at
  *       k + s*k_stride_seq + (seq_start[s] + i)*k_stride_tok + g*k_stride_head
  *     (strides in elements, head_dim contiguous); V likewise.  Rows
@@ -102,8 +111,11 @@ refree_status refree_score(const refree_params *p, const void *q_win, const void
                            int32_t *device_status, void *stream);
 
 /* Steps S4-S6: rank the positions, evaluate the stopping rule (Eq. 1 / Eq. 3;
- * Algorithm 1 Square .. Where) in fp64 over the squares of the fp32 scores,
- * apply the window floor, and emit the kept set in ascending position order.
+ * Algorithm 1 Square .. Where) over the exact squares of the fp32 scores: the
+ * 48-bit squared mantissas are summed as integers in a per-unit fixed point
+ * (order-independent, so budgets are deterministic) and the crossing level
+ * (1 - T)^2 C_n is evaluated once in fp64; then apply the window floor and emit
+ * the kept set in ascending position order.
  *   lengths  [num_seqs * num_kv_heads] int32
  *   offsets  [num_seqs * num_kv_heads + 1] int64, running sum of lengths
  *   kept_idx [capacity_rows] int32 positions within their sequence (nullable:

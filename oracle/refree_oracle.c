@@ -22,8 +22,8 @@
  *                    for the score ranking.
  *   oracle_compact - row-by-row byte comparison against numpy fancy indexing.
  *
- * Readings of the paper taken here (each is listed with its reason in the
- * design notes):
+ * Readings of the paper taken here, where it is silent, garbled or at odds
+ * with itself:
  *   - Eq. 2: column i of the last w rows of A, divided by the number of those
  *     rows that can see i causally, min(w_eff, n - i).
  *   - Eq. 1 / Eq. 3: leftmost j with 1 - sqrt(C_j / C_n) < T, strict; the kept

@@ -77,20 +77,28 @@ compact_kernel(refree_params p, const char *k, const char *v, const int32_t *seq
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     for (int64_t e0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; e0 < nvec; e0 += stride * kUnroll) {
         int4 kv[kUnroll], vv[kUnroll];
+        bool good[kUnroll];
 #pragma unroll
         for (int r = 0; r < kUnroll; ++r) {
             const int64_t e = e0 + r * stride;
+            good[r] = false;
             if (e < nvec) {
                 const int t = (int)(e >> vshift), c = (int)(e & (vec_per_row - 1));
                 const int src = position_ranges ? (t < head ? t : n - b + t) : idx[t];
-                kv[r] = *reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok + c * 16);
-                vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16));
+                // an index list is the caller's: a row outside the sequence is reported, never read
+                good[r] = src >= 0 && src < n;
+                if (good[r]) {
+                    kv[r] = *reinterpret_cast<const int4 *>(kb + (int64_t)src * k_tok + c * 16);
+                    vv[r] = ld_stream(reinterpret_cast<const int4 *>(vb + (int64_t)src * v_tok + c * 16));
+                } else if (dev_status) {
+                    atomicOr(dev_status, REFREE_DEV_CAPACITY);
+                }
             }
         }
 #pragma unroll
         for (int r = 0; r < kUnroll; ++r) {
             const int64_t e = e0 + r * stride;
-            if (e < nvec) {
+            if (e < nvec && good[r]) {
                 st_stream(reinterpret_cast<int4 *>(ko + e * 16), kv[r]);
                 st_stream(reinterpret_cast<int4 *>(vo + e * 16), vv[r]);
             }
@@ -317,14 +325,14 @@ cudaError_t launch_compact(const refree_params &p, const void *k, const void *v,
         // registers each): 10 240 registers are left per SM, so the block is 128 threads (8 192
         // registers), and the grid is many short-lived blocks, so that a scoring CTA that becomes
         // runnable finds room as soon as a few of them retire.
-        const int gx = max(1, (148 * 32) / U);
+        const int gx = max(1, (sm_count() * 32) / U);
         compact_kernel<kThreadsSlim><<<dim3(gx, U), kThreadsSlim, 0, st>>>(
             p, (const char *)k, (const char *)v, seq_start, seq_len, lengths, offsets, kept_idx,
             position_ranges ? 1 : 0, offsets_out, (char *)k_out, (char *)v_out, capacity_rows, dev_status);
         count_launches(1);
         return cudaGetLastError();
     }
-    const int gx = max(1, (148 * 8) / U);
+    const int gx = max(1, (sm_count() * 8) / U);
     compact_kernel<kThreads><<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
                                                      lengths, offsets, kept_idx, position_ranges ? 1 : 0, offsets_out,
                                                      (char *)k_out, (char *)v_out, capacity_rows, dev_status);
@@ -376,7 +384,7 @@ cudaError_t launch_compact_paged(const refree_params &p, const void *k, const vo
                                  int64_t num_blocks, int32_t *dev_status, cudaStream_t st)
 {
     const int U = p.num_seqs * p.num_kv_heads;
-    const int gx = max(1, (148 * 8) / U);
+    const int gx = max(1, (sm_count() * 8) / U);
     compact_paged_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, (const char *)k, (const char *)v, seq_start, seq_len,
                                                            lengths, offsets, kept_idx, position_ranges ? 1 : 0,
                                                            block_table, max_blocks_per_unit, block_rows,

@@ -514,7 +514,7 @@ cudaError_t run_mma(const DecArgs &a, dim3 grid, int G, cudaStream_t st)
 void decode_shape(const refree_params &p, int64_t max_rows, int &gx, int &span)
 {
     const int64_t U = (int64_t)p.num_seqs * p.num_kv_heads;
-    const int64_t want = std::max<int64_t>(1, 148 / U);   // about one block per SM (one wave: prologue and merge are paid once)
+    const int64_t want = std::max<int64_t>(1, sm_count() / U);   // about one block per SM (one wave: prologue and merge are paid once)
     const int64_t by_rows = std::max<int64_t>(1, (max_rows + 127) / 128);      // at least one 16-row block per warp
     gx = (int)std::min<int64_t>(want, by_rows);
     span = (int)(((max_rows + gx - 1) / gx + 15) / 16 * 16);

@@ -60,6 +60,9 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens);
 // Bookkeeping for refree_kernel_launch_count(): every launcher adds the kernels it enqueued.
 void count_launches(int n);
 
+// Multiprocessors of the current device (looked up once per device; launch geometry is sized by it).
+int sm_count();
+
 inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Per-CTA tables: running sums of sequence lengths and of tiles per sequence.

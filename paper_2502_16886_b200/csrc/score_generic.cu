@@ -203,7 +203,7 @@ cudaError_t run(const refree_params &p, const void *q_win, const void *k, const 
     e = cudaFuncSetAttribute(score_colsum_generic<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t max_items = (total_tokens / kTile + p.num_seqs) * p.num_kv_heads;
-    const int grid = (int)std::min<int64_t>(std::max<int64_t>(max_items, 1), 148 * 16);
+    const int grid = (int)std::min<int64_t>(std::max<int64_t>(max_items, 1), sm_count() * 16);
     float2 *part = reinterpret_cast<float2 *>(ws + lay.part_off);
     float *lse = reinterpret_cast<float *>(ws + lay.lse_off);
     score_stats_generic<T, D><<<grid, kThreads, smem, st>>>(p, (const T *)q_win, (const T *)k, seq_start, seq_len, part);

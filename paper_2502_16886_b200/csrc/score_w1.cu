@@ -417,12 +417,11 @@ w1_scores_kernel(W1Args a)
     }
 }
 
-constexpr int kScoreGrid = 148 * 4;
 
 template <int GMAX>
 cudaError_t run_w1_scores(W1Args &a, int64_t chunk_items, cudaStream_t st)
 {
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(chunk_items, kScoreGrid));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(chunk_items, sm_count() * 4));
     w1_scores_kernel<GMAX><<<grid, kThreadsW1, 0, st>>>(a);
     count_launches(1);
     return cudaGetLastError();
@@ -491,17 +490,17 @@ cudaError_t launch_score_w1(const refree_params &p, const void *q_win, const voi
     if (!f32 && !(reinterpret_cast<uintptr_t>(q_win) & 15)) {
         // one span per warp when the pass fits a single wave of 2 blocks per SM; capped so that
         // short sequences still spread over the machine
-        const int64_t warps = 148 * 2 * (kThreadsW1 / 32);
+        const int64_t warps = (int64_t)sm_count() * 2 * (kThreadsW1 / 32);
         const int64_t rows = total_tokens * p.num_kv_heads;
         int64_t span = (rows + warps - 1) / warps;
         span = std::min<int64_t>(kMaxSpan, std::max<int64_t>(kMinSpan, (span + 15) / 16 * 16));
         a.span = (int)span;
         const int64_t span_items = (total_tokens / span + p.num_seqs) * p.num_kv_heads;
-        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((span_items + 7) / 8, 148 * 2));
+        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((span_items + 7) / 8, sm_count() * 2));
         e = p.head_dim == 64 ? run_w1_mma<64>(a, q_win, k, grid, st, G) : run_w1_mma<128>(a, q_win, k, grid, st, G);
     } else {
         a.span = kChunk;
-        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(chunk_items, 148 * 8));
+        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(chunk_items, sm_count() * 8));
         if (p.head_dim == 64)
             e = f32 ? run_w1_lanes<float, 64>(a, q_win, k, grid, st, G) : run_w1_lanes<__nv_bfloat16, 64>(a, q_win, k, grid, st, G);
         else

@@ -45,7 +45,7 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     w.part_off = off;   w.part_bytes = align256(part_bytes);                                               off += w.part_bytes;
     w.lse_off = off;    w.lse_bytes = align256((size_t)(U * rows_pad) * sizeof(float));                    off += w.lse_bytes;
     w.grp_off = off;    w.grp_bytes = align256((size_t)(tiles * p.num_kv_heads * 4) * sizeof(GroupPartial));  off += w.grp_bytes;
-    w.cnt_off = off;    w.cnt_bytes = align256((size_t)(U + 256 + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
+    w.cnt_off = off;    w.cnt_bytes = align256((size_t)(2 * U + 256 + 8) * sizeof(int32_t));                         off += w.cnt_bytes;
     w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
     w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
     w.kept_off = off;   w.kept_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(int32_t)); off += w.kept_bytes;
@@ -502,6 +502,7 @@ refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
             t.ws = ws;
             t.scores = reinterpret_cast<float *>(ws + lay.scores_off);
             t.groups = p->scope == REFREE_SCOPE_HEAD ? reinterpret_cast<GroupPartial *>(ws + lay.grp_off) : nullptr;
+            t.sel_lengths = t.groups ? lengths[l] : nullptr;      // the rule runs inside the launch that finishes the layer
             return t;
         };
         auto job_of = [&](int l) {
@@ -523,9 +524,9 @@ refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
             if (j >= 1) fin = layer_of(j - 1);
             if (j >= 2) job = job_of(j - 2);
             if (launch_score_tc_pipe(*p, j < num_layers ? &beg : nullptr, j >= 1 ? &fin : nullptr, seq_start, seq_len,
-                                     total_tokens, lay, device_status, cs, j >= 2 ? &job : nullptr) != cudaSuccess)
+                                     total_tokens, lay, device_status, cs, j >= 2 ? &job : nullptr, true) != cudaSuccess)
                 return REFREE_ERR_CUDA;
-            if (j >= 1 &&
+            if (j >= 1 && !fin.sel_lengths &&
                 launch_select(*p, fin.scores, seq_len, total_tokens, lengths[j - 1], offsets[j - 1], nullptr, capacity_rows,
                               fin.ws, lay, device_status, cs, false, fin.groups) != cudaSuccess)
                 return REFREE_ERR_CUDA;

@@ -156,13 +156,16 @@ struct TcLayer {
     float *scores;          // [Hkv, total_tokens]
     char *ws;               // the layer's workspace (partials between its two passes)
     GroupPartial *groups;   // nullable
+    int32_t *sel_lengths;   // nullable: with `groups`, the launch that finishes the layer also evaluates the stopping
+                            // rule (position ranking per head) and leaves the budgets here
 };
 // One launch of a run: the column pass of `finish`, then the row pass of `begin` (either may be null), and the
-// rows of `copy` (nullable) moved beside them.
+// rows of `copy` (nullable) moved beside them.  A launch clears the per-unit tile counts that the launch finishing
+// its `begin` layer will use; `finish_tickets_clean` says an earlier launch of the run did that for this one.
 cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, const TcLayer *finish,
                                  const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
                                  const Workspace &lay, int32_t *dev_status, cudaStream_t st,
-                                 const TcCopyJob *copy = nullptr);
+                                 const TcCopyJob *copy = nullptr, bool finish_tickets_clean = false);
 
 // Single query row per head (the paper's default reduced attention): a stream over K on the fp32 pipes.
 bool score_w1_supported(const refree_params &p);

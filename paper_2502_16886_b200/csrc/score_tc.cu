@@ -37,13 +37,14 @@
 #include <mutex>
 
 #include "refree_internal.cuh"
+#include "select_groups.cuh"
 
 namespace refree {
 namespace {
 
 constexpr int kEpiWarps = 16;
-constexpr int kThreadsTc = (kEpiWarps + 3) * 32;    // + TMA warp, MMA warp, copy warp
-constexpr int kMaxCopySlots = 6;
+constexpr int kThreadsTc = (kEpiWarps + 4) * 32;    // + TMA warp, MMA warp, copy warp, finishing warp
+constexpr int kMaxCopySlots = 10;
 constexpr int kMaxCopyUnits = 1024;                 // units whose running budget sum fits the CTA's table
 constexpr int kD = 128;
 constexpr int kCopyRows = 32;                       // rows of one piece of the in-kernel row copy
@@ -220,13 +221,14 @@ constexpr int kInfoRing = 16;   // the TMA thread runs at most ring stages + acc
 struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
     uint64_t acc_full[4], acc_empty[4];       // pass 1: accumulator (pair * 2 + slot), 128 tensor-memory columns each
-    uint64_t p2_full[2], p2_empty[2];         // pass 2: accumulators of 256 columns
-    uint64_t chunk_ready[4];                  // pass 2: the other column chunks have staged their shares of a tile
+    uint64_t p2_full[2], p2_empty[2];         // pass 2: accumulators of 256 columns, one per group of eight warps
+    uint64_t chunk_ready[4];                  // pass 2: every share of a tile has been staged
+    uint64_t stage_free[4];                   // pass 2: the finishing warp has read the slot
     uint64_t c_full[kMaxCopySlots];           // row copy: a piece has landed in its slot
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) ItemInfo info[kInfoRing];
-    alignas(16) float stage[4][3][kTile];     // pass 2: partial column sums of chunks 1..3, four tiles deep
+    alignas(16) float stage[4][4][kTile];     // pass 2: partial column sums (share = product * 2 + column half), four tiles deep
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
 };
 
@@ -301,6 +303,12 @@ struct TcArgs {
     uint32_t *flags;     // one layer per launch: flags[c] != 0 once CTA c has written its pass-1 partials (zeroed before the launch)
     int64_t total_tokens;
     int32_t *dev_status;
+    // Stopping rule inside the launch (position ranking per head): the finishing warp that completes a unit's
+    // last tile (a ticket per unit) evaluates the rule from the unit's records.  All nullable.
+    int32_t *sel_lengths;      // [units] budgets out
+    Cut *sel_cuts;             // [units]
+    uint32_t *tickets;         // [2 units] tiles finished per unit, then the unit's largest score; zero when the launch begins
+    uint32_t *tickets_next;    // [2 units] those of the launch that follows, cleared by this one
     TcCopyJob cj;          // rows of an earlier layer to move while this layer is scored (nslots == 0: none)
 };
 
@@ -658,47 +666,34 @@ __device__ inline void col_sum16(const uint32_t (&cur)[32], float scale, const f
     }
 }
 
-template <int WIDTH, bool MASKED>
-__device__ inline float col_job(uint32_t taddr, uint64_t *empty_bar, int lane, float scale, const float *lse,
+// One product's share of a warp: `nch` chunks of 16 columns (rows of Q) come from tensor memory one chunk at a
+// time, the next in flight while 2^(y - L[row]) is summed over the current one; the accumulator is handed back
+// as soon as the last load has landed.
+template <bool MASKED>
+__device__ inline float col_job(int nch, uint32_t taddr, uint64_t *empty_bar, int lane, float scale, const float *lse,
                                 int rbase, int R, int w, int pos_gap)
 {
-    constexpr int NCH = WIDTH / 16;
     uint32_t b0[32], b1[32];               // only the first 16 of each are used
     float s0 = 0.f, s1 = 0.f;
-    tmem_ld16_issue(taddr, b0);
-    tmem_ld_wait16(b0);
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-        uint32_t (&cur)[32] = (c & 1) ? b1 : b0;
-        uint32_t (&nxt)[32] = (c & 1) ? b0 : b1;
-        if (c + 1 < NCH) tmem_ld16_issue(taddr + 16 * (c + 1), nxt);
-        if (c + 1 == NCH) {
-            // every load has landed
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar);
-        }
-        col_sum16<MASKED>(cur, scale, lse, rbase + 16 * c, R, w, pos_gap, s0, s1);
-        if (c + 1 < NCH) tmem_ld_wait16(nxt);
-    }
-    return s0 + s1;
-}
-
-template <bool MASKED>
-__device__ inline float col_job_any(int width, uint32_t taddr, uint64_t *empty_bar, int lane, float scale,
-                                    const float *lse, int rbase, int R, int w, int pos_gap)
-{
-    switch (width) {
-    case 64: return col_job<64, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
-    case 48: return col_job<48, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
-    case 32: return col_job<32, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
-    case 16: return col_job<16, MASKED>(taddr, empty_bar, lane, scale, lse, rbase, R, w, pos_gap);
-    default:
+    auto release = [&]() {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar);
-        return 0.f;
+    };
+    if (nch <= 0) { release(); return 0.f; }
+    tmem_ld16_issue(taddr, b0);
+    tmem_ld_wait16(b0);
+    for (int c = 0; c < nch; c += 2) {
+        if (c + 1 < nch) tmem_ld16_issue(taddr + 16 * (c + 1), b1); else release();
+        col_sum16<MASKED>(b0, scale, lse, rbase + 16 * c, R, w, pos_gap, s0, s1);
+        if (c + 1 < nch) {
+            tmem_ld_wait16(b1);
+            if (c + 2 < nch) tmem_ld16_issue(taddr + 16 * (c + 2), b0); else release();
+            col_sum16<MASKED>(b1, scale, lse, rbase + 16 * (c + 1), R, w, pos_gap, s0, s1);
+            if (c + 2 < nch) tmem_ld_wait16(b0);
+        }
     }
+    return s0 + s1;
 }
 
 // CTA that owns item x when `items` are split evenly over `ctas` (ctas <= items).
@@ -707,160 +702,218 @@ __device__ inline int cta_of_item(int x, int items, int ctas)
     return (int)((((int64_t)x + 1) * ctas - 1) / items);
 }
 
+// L[row] = log2 sum over the row of 2^y for the rows of unit u, merged from the (reference, sum) pairs that pass 1
+// left per (CTA, unit, column half), in ascending record order (the same in every CTA that needs the unit).
+// Called by all epilogue threads; `ib` = index of the unit's first item, `ts` = its tiles.
+__device__ inline bool merge_unit_lse(const TcArgs &a, TcSmemTail &tl, int u, int ib, int ts, int items, int ctas,
+                                      uint32_t &ephase)
+{
+    const TcShape &sh = a.sh;
+    const int tid = threadIdx.x;
+    const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
+    if (a.flags) {
+        // one launch for both passes: the partials of this unit come from CTAs that may still be in pass 1;
+        // wait (bounded) until each of them has published
+        for (int c = c_lo + tid; c <= c_hi; c += kEpiWarps * 32) {
+            bool seen = false;
+            for (uint32_t spin = 0; spin < kSpinLimit && !seen; ++spin) {
+                uint32_t v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.flags + c) : "memory");
+                seen = v != 0u;
+                if (!seen) { if (tl.abort_flag) break; __nanosleep(spin > 64 ? 256 : 32); }
+            }
+            if (!seen) tl.abort_flag = 1;
+        }
+        if (!epi_sync(tl, ephase)) return false;
+        if (tl.abort_flag) return false;
+    }
+    // two threads per row when there are enough threads: even and odd records, then one exchange
+    const int per_row = 2 * sh.R <= kEpiWarps * 32 ? 2 : 1;
+    const int r = tid / per_row, sub = tid % per_row;
+    float M = -INFINITY, Z = 0.f;
+    if (r < sh.R) {
+        const int s_hi = 2 * (c_hi + u) + 1;               // records: (CTA, column half)
+        constexpr int kBatch = 12;                          // independent loads in flight per thread
+        for (int s0 = 2 * (c_lo + u) + sub; s0 <= s_hi; s0 += kBatch * per_row) {
+            float2 pr[kBatch];
+#pragma unroll
+            for (int q = 0; q < kBatch; ++q)
+                pr[q] = (s0 + q * per_row <= s_hi) ? __ldcg(&a.part_b[(int64_t)(s0 + q * per_row) * sh.Rpad + r])
+                                                   : make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int q = 0; q < kBatch; ++q) {
+                if (pr[q].y > 0.f) {
+                    if (pr[q].x > M) { Z = Z * ex2(M - pr[q].x) + pr[q].y; M = pr[q].x; }
+                    else Z += pr[q].y * ex2(pr[q].x - M);
+                }
+            }
+        }
+    }
+    if (per_row == 2) {
+        const float M2 = __shfl_xor_sync(0xffffffffu, M, 1), Z2 = __shfl_xor_sync(0xffffffffu, Z, 1);
+        // (even records) then (odd records), in that order on both lanes
+        const float Ma = sub ? M2 : M, Za = sub ? Z2 : Z, Mb = sub ? M : M2, Zb = sub ? Z : Z2;
+        if (Zb > 0.f) {
+            if (Za > 0.f) {
+                if (Mb > Ma) { Z = Za * ex2(Ma - Mb) + Zb; M = Mb; }
+                else { Z = Za + Zb * ex2(Mb - Ma); M = Ma; }
+            } else { Z = Zb; M = Mb; }
+        } else { Z = Za; M = Ma; }
+    }
+    // a row that sees nothing adds 2^(-inf) = 0
+    if (r < sh.R && sub == 0) tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;
+    // columns past the unit's rows (padding of the last product) never count
+    for (int rr = sh.R + tid; rr < sh.cblocks * sh.ncol; rr += kEpiWarps * 32) tl.lse[rr] = INFINITY;
+    return epi_sync(tl, ephase);
+}
+
+// Pass 2, the sixteen epilogue warps.  Two groups of eight warps take the products in turn (product j goes to
+// group j & 1 and to accumulator j & 1), so the groups run out of step: while one waits for its next accumulator,
+// stages a tile or refills its pipeline, the other keeps the exponential units busy.  Inside a group a warp is
+// (lane quarter) x (half of the product's columns); it leaves its share of the tile's column sums in a staging
+// slot, and the finishing warp adds the shares.
 __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const SeqView &sv, uint32_t tmem_base,
-                                      int nitems, int items, int ctas, EpiState &es)
+                                      int item0, int nitems, int items, int ctas, EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int chunk = warp >> 2;                                   // 0 finishes the tile, 1..3 stage their shares
+    const int group = (warp >> 2) & 1, half = warp >> 3;
     const int lane_base = (warp & 3) * 32;
-    const int tid = threadIdx.x;                                   // 0..511
     const float scale = kLog2e * rsqrtf((float)kD);
     const int w = a.p.window;
     const int pos_in_tile = lane_base + lane;
-    // this warp's columns of a product: whole groups of 16, split as evenly as the four chunks allow
-    const int units16 = sh.ncol >> 4;
-    const int c_begin = (chunk * units16 / 4) * 16, c_width = ((chunk + 1) * units16 / 4) * 16 - c_begin;
+    const int c_width = sh.ncol >> 1, c_begin = half * c_width;     // this warp's columns of a product
     const bool exact = sh.cblocks * sh.ncol == sh.R;               // no padding columns in the products
-    uint32_t cnt = 0;                                              // products consumed
     uint32_t &ephase = es.ephase;                                  // phase of the epilogue barrier
-    uint32_t tcount = 0;                                           // tiles seen
-    // chunk 0 finishes a tile one tile late, when the other chunks' shares have long been staged
-    float pend_acc = 0.f;
-    const ItemInfo *pend_inf = nullptr;        // the pending tile's record (still in the ring: it is one item old)
+    uint32_t gcnt = 0;                                             // products this group has taken
+    int next_change = 0;                                           // item (relative) at which the next unit begins
     bool ok = true;
-    auto finish_pending = [&]() -> bool {
-        if (!pend_inf) return true;
-        const uint32_t pend_tile = tcount - 1u;
-        float tot = pend_acc;
-        if (!mbar_wait(&tl.chunk_ready[pend_tile & 3u], (pend_tile >> 2) & 1u, &tl.abort_flag)) return false;
-        tot += tl.stage[pend_tile & 3u][0][pos_in_tile];
-        tot += tl.stage[pend_tile & 3u][1][pos_in_tile];
-        tot += tl.stage[pend_tile & 3u][2][pos_in_tile];
-        const int n = pend_inf->n, i = pend_inf->tile * kTile + pos_in_tile;
-        const int G = a.p.num_q_heads / a.p.num_kv_heads;
-        const int cnt_i = max(1, min(min(w, n), n - i));
-        float sc = 0.f;
-        if (i < n) {
-            sc = tot / ((float)cnt_i * (float)G);
-            if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
-            a.scores[(int64_t)pend_inf->g * a.total_tokens + pend_inf->pack + i] = sc;
-        }
-        if (a.groups) {
-            // this warp's 32 positions: largest score, and the exact squares summed at a scale set by it
-            const uint32_t bits = (i < n && isfinite(sc)) ? mag_bits(sc) : 0u;
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, bits);
-            unsigned long long sq = sq_fixed(bits, kGroupShift - 2 * max(1, (int)(mx >> 23)));
-            for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-            if (lane == 0) {
-                GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq;
-                a.groups[((int64_t)pend_inf->ib + pend_inf->tile) * 4 + (warp & 3)] = gp;
-            }
-        }
-        pend_inf = nullptr;
-        return true;
-    };
     for (int item = 0; item < nitems && ok; ++item) {
         const ItemInfo *inf = &tl.info[es.icount++ & (kInfoRing - 1)];
-        float accv = 0.f;
-        int tile_start = 0, n = 0;
-        for (int cb = 0; cb < sh.cblocks && ok; ++cb) {
-            const int buf = (int)(cnt & 1u);
-            ok = mbar_wait(&tl.p2_full[buf], (cnt >> 1) & 1u, &tl.abort_flag);
+        if (item == next_change) {
+            // A unit begins: all sixteen warps meet (the two groups share L), whichever group takes the item's
+            // products.  The unit is looked up in the sequence tables, not in the item's record, which a warp
+            // that takes none of the item's products has no barrier to wait for.  The normalisers do not wait
+            // for the tile either: the partials come from the row pass, not from anything this pass loads.
+            const ItemTc it = decode_item_tc(sv, a.p.num_seqs, a.p.num_kv_heads, item0 + item);
+            if (item > 0 && !(ok = epi_sync(tl, ephase))) break;   // nobody still reads the previous unit's L
+            ok = merge_unit_lse(a, tl, it.u, sv.tiles[it.s] * a.p.num_kv_heads + it.g * it.ntiles, it.ntiles, items, ctas,
+                                ephase);
             if (!ok) break;
-            ++cnt;
+            next_change = item + (it.ntiles - it.tile);
+        }
+        for (int cb = 0; cb < sh.cblocks && ok; ++cb) {
+            const uint32_t j = (uint32_t)item * (uint32_t)sh.cblocks + (uint32_t)cb;      // product index in this pass
+            if ((int)(j & 1u) != group) continue;
+            ok = mbar_wait(&tl.p2_full[group], gcnt & 1u, &tl.abort_flag);
+            if (!ok) break;
+            ++gcnt;
             tc_fence_after();
-            if (cb == 0) {
-                // the item's record is valid from the item's first product on
-                if (inf->new_unit) {
-                    if (!(ok = epi_sync(tl, ephase))) break;       // nobody still reads the previous unit's L
-                    // L[row] = log2 sum over the row of 2^y, merged from the (reference, sum) pairs that pass 1
-                    // left per (CTA, unit), in ascending CTA order (the same order in every CTA that needs it)
-                    const int u = inf->u, ts = inf->ntiles, ib = inf->ib;
-                    const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
-                    if (a.flags) {
-                        // one launch for both passes: the partials of this unit come from CTAs that may still be
-                        // in pass 1; wait (bounded) until each of them has published
-                        for (int c = c_lo + tid; c <= c_hi; c += kEpiWarps * 32) {
-                            bool seen = false;
-                            for (uint32_t spin = 0; spin < kSpinLimit && !seen; ++spin) {
-                                uint32_t v;
-                                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.flags + c) : "memory");
-                                seen = v != 0u;
-                                if (!seen) { if (tl.abort_flag) break; __nanosleep(spin > 64 ? 256 : 32); }
-                            }
-                            if (!seen) tl.abort_flag = 1;
-                        }
-                        if (!(ok = epi_sync(tl, ephase))) break;
-                        if (tl.abort_flag) { ok = false; break; }
-                    }
-                    // two threads per row when there are enough threads: even and odd records, then one exchange
-                    const int per_row = 2 * sh.R <= kEpiWarps * 32 ? 2 : 1;
-                    const int r = tid / per_row, sub = tid % per_row;
-                    float M = -INFINITY, Z = 0.f;
-                    if (r < sh.R) {
-                        const int s_hi = 2 * (c_hi + u) + 1;               // records: (CTA, column half)
-                        for (int s0 = 2 * (c_lo + u) + sub; s0 <= s_hi; s0 += 8 * per_row) {
-                            float2 pr[8];                                  // eight independent loads in flight
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                pr[q] = (s0 + q * per_row <= s_hi)
-                                            ? __ldcg(&a.part_b[(int64_t)(s0 + q * per_row) * sh.Rpad + r])
-                                            : make_float2(-INFINITY, 0.f);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                if (pr[q].y > 0.f) {
-                                    if (pr[q].x > M) { Z = Z * ex2(M - pr[q].x) + pr[q].y; M = pr[q].x; }
-                                    else Z += pr[q].y * ex2(pr[q].x - M);
-                                }
-                            }
-                        }
-                    }
-                    if (per_row == 2) {
-                        const float M2 = __shfl_xor_sync(0xffffffffu, M, 1), Z2 = __shfl_xor_sync(0xffffffffu, Z, 1);
-                        // (even records) then (odd records), in that order on both lanes
-                        const float Ma = sub ? M2 : M, Za = sub ? Z2 : Z, Mb = sub ? M : M2, Zb = sub ? Z : Z2;
-                        if (Zb > 0.f) {
-                            if (Za > 0.f) {
-                                if (Mb > Ma) { Z = Za * ex2(Ma - Mb) + Zb; M = Mb; }
-                                else { Z = Za + Zb * ex2(Mb - Ma); M = Ma; }
-                            } else { Z = Zb; M = Mb; }
-                        } else { Z = Za; M = Ma; }
-                    }
-                    // a row that sees nothing adds 2^(-inf) = 0
-                    if (r < sh.R && sub == 0) tl.lse[r] = Z > 0.f ? M + log2f(Z) : INFINITY;
-                    // columns past the unit's rows (padding of the last product) never count
-                    for (int rr = sh.R + tid; rr < sh.cblocks * sh.ncol; rr += kEpiWarps * 32) tl.lse[rr] = INFINITY;
-                    if (!(ok = epi_sync(tl, ephase))) break;
-                }
-                tile_start = inf->tile * kTile;
-                n = inf->n;
-            }
+            // the item's record is valid once one of its products is
+            const int tile_start = inf->tile * kTile, n = inf->n;
             const int pos_gap = tile_start + pos_in_tile - (n - w);
             // tile wholly before the window and wholly inside the sequence: every row sees every position
             const bool full = tile_start + kTile <= n - w + 1 && exact;
-            const uint32_t taddr = tmem_base + (uint32_t)buf * 256u + (uint32_t)c_begin + ((uint32_t)lane_base << 16);
-            accv += full ? col_job_any<false>(c_width, taddr, &tl.p2_empty[buf], lane, scale, tl.lse, cb * sh.ncol + c_begin,
-                                              sh.R, w, pos_gap)
-                         : col_job_any<true>(c_width, taddr, &tl.p2_empty[buf], lane, scale, tl.lse, cb * sh.ncol + c_begin,
-                                             sh.R, w, pos_gap);
-        }
-        if (!ok) break;
-        // Chunk 0 completes the previous tile only now, so its wait for the other chunks' shares of that
-        // tile has long been satisfied.  The others can be at most three tiles past the staging slot read
-        // here (an accumulator is handed back by all sixteen warps, chunk 0 included): four slots.
-        if (chunk == 0) {
-            if (!(ok = finish_pending())) break;
-            pend_acc = accv;
-            pend_inf = inf;
-        } else {
-            tl.stage[tcount & 3u][chunk - 1][pos_in_tile] = accv;
+            const uint32_t taddr = tmem_base + (uint32_t)group * 256u + (uint32_t)c_begin + ((uint32_t)lane_base << 16);
+            const float part = full ? col_job<false>(c_width >> 4, taddr, &tl.p2_empty[group], lane, scale, tl.lse,
+                                                     cb * sh.ncol + c_begin, sh.R, w, pos_gap)
+                                    : col_job<true>(c_width >> 4, taddr, &tl.p2_empty[group], lane, scale, tl.lse,
+                                                    cb * sh.ncol + c_begin, sh.R, w, pos_gap);
+            // the slot's previous tile (four tiles ago) has been read by the finishing warp
+            const uint32_t slot = (uint32_t)item & 3u;
+            if (!(ok = mbar_wait(&tl.stage_free[slot], (((uint32_t)item >> 2) & 1u) ^ 1u, &tl.abort_flag))) break;
+            tl.stage[slot][cb * 2 + half][pos_in_tile] = part;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tl.chunk_ready[tcount & 3u]);
+            if (lane == 0) mbar_arrive(&tl.chunk_ready[slot]);
         }
-        ++tcount;
     }
-    if (chunk == 0 && ok) finish_pending();
+}
+
+// Pass 2, the finishing warp: a'[i] = (sum of the warps' shares, in a fixed order) / (G * rows that see i)  (Eq. 2), the score
+// store, and per 32 positions the record the stopping rule reads.  `icount0` = items the roles have gone through
+// before this pass (their ring index).
+__device__ inline void finisher_pass2(const TcArgs &a, TcSmemTail &tl, int nitems, uint32_t icount0)
+{
+    const int lane = threadIdx.x & 31;
+    const int w = a.p.window;
+    const float g = (float)(a.p.num_q_heads / a.p.num_kv_heads);
+    const bool two_products = a.sh.cblocks > 1;
+    // This CTA's tiles of a unit are counted once, when its run of them ends: the warp that brings the unit's count
+    // to its number of tiles sees every other tile's scores and records (fenced before their counts were added)
+    // and evaluates the stopping rule for the unit.
+    int run_u = -1, run_n = 0, run_ntiles = 0, run_ib = 0, run_tiles = 0;
+    uint32_t run_max = 0;                       // largest score of the run (bit pattern)
+    const float *run_dst = nullptr;
+    const int U = a.p.num_seqs * a.p.num_kv_heads;
+    auto close_run = [&]() {
+        if (run_u < 0 || run_tiles == 0) return;
+        if (lane == 0) atomicMax(&a.tickets[U + run_u], run_max);      // the unit's largest score, beside its count
+        __threadfence();
+        __syncwarp();
+        uint32_t old = 0;
+        if (lane == 0) old = atomicAdd(&a.tickets[run_u], (uint32_t)run_tiles);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if ((int)old + run_tiles == run_ntiles) {
+            __threadfence();
+            uint32_t umax = 0;
+            if (lane == 0) umax = atomicMax(&a.tickets[U + run_u], 0u);
+            umax = __shfl_sync(0xffffffffu, umax, 0);
+            const Cut cut = select_unit_from_groups_warp(a.p, run_dst, run_n, a.groups + (int64_t)run_ib * 4, umax);
+            if (lane == 0) {
+                a.sel_lengths[run_u] = cut.b;
+                if (a.sel_cuts) a.sel_cuts[run_u] = cut;
+            }
+        }
+        run_tiles = 0;
+    };
+    for (int t = 0; t < nitems; ++t) {
+        const uint32_t slot = (uint32_t)t & 3u;
+        if (!mbar_wait(&tl.chunk_ready[slot], ((uint32_t)t >> 2) & 1u, &tl.abort_flag)) return;
+        const ItemInfo *inf = &tl.info[(icount0 + (uint32_t)t) & (kInfoRing - 1)];
+        const int n = inf->n, tile = inf->tile;
+        const int inf_u = inf->u, inf_ntiles = inf->ntiles, inf_ib = inf->ib;     // the record may be reused after the slot is freed
+        float *dst = a.scores + (int64_t)inf->g * a.total_tokens + inf->pack;
+        GroupPartial *grp = a.groups ? a.groups + ((int64_t)inf->ib + tile) * 4 : nullptr;
+        uint32_t tile_max = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int pos = q * 32 + lane, i = tile * kTile + pos;
+            float tot = tl.stage[slot][0][pos];
+            tot += tl.stage[slot][1][pos];
+            if (two_products) {
+                tot += tl.stage[slot][2][pos];
+                tot += tl.stage[slot][3][pos];
+            }
+            const int cnt_i = max(1, min(min(w, n), n - i));
+            float sc = 0.f;
+            if (i < n) {
+                sc = tot / ((float)cnt_i * g);
+                if (!isfinite(sc) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
+                dst[i] = sc;
+            }
+            if (grp) {
+                // these 32 positions: largest score, and the exact squares summed at a scale set by it
+                const uint32_t bits = (i < n && isfinite(sc)) ? mag_bits(sc) : 0u;
+                const uint32_t mx = __reduce_max_sync(0xffffffffu, bits);
+                tile_max = max(tile_max, mx);
+                unsigned long long sq = sq_fixed(bits, kGroupShift - 2 * max(1, (int)(mx >> 23)));
+                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (lane == 0) { GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq; grp[q] = gp; }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tl.stage_free[slot]);
+        if (a.tickets) {
+            if (inf_u != run_u) {
+                close_run();
+                run_u = inf_u; run_n = n; run_ntiles = inf_ntiles; run_ib = inf_ib; run_dst = dst; run_tiles = 0;
+                run_max = 0;
+            }
+            ++run_tiles;
+            run_max = max(run_max, tile_max);
+        }
+    }
+    if (a.tickets) close_run();
 }
 
 // ------------------------------------------------------------- row copy -----
@@ -1016,13 +1069,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         mbar_init(&tl.q_full, 1);
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tl.p2_full[b], 1); mbar_init(&tl.p2_empty[b], kEpiWarps); }
-        for (int b = 0; b < 4; ++b) mbar_init(&tl.chunk_ready[b], 12);      // the twelve warps of chunks 1..3
+        for (int b = 0; b < 2; ++b) { mbar_init(&tl.p2_full[b], 1); mbar_init(&tl.p2_empty[b], kEpiWarps / 2); }
+        for (int b = 0; b < 4; ++b) {
+            mbar_init(&tl.chunk_ready[b], (kEpiWarps / 2) * a.sh.cblocks);      // eight warps stage a share per product
+            mbar_init(&tl.stage_free[b], 1);
+        }
         mbar_init(&tl.epi_bar, kEpiWarps);
         for (int b = 0; b < kMaxCopySlots; ++b) mbar_init(&tl.c_full[b], 1);
         tl.abort_flag = 0;
         fence_barrier_init();
     }
+    if (a.tickets_next && blockIdx.x == 0)
+        for (int t = threadIdx.x; t < 2 * B * a.p.num_kv_heads; t += kThreadsTc) a.tickets_next[t] = 0u;
+    if (a.sel_lengths && blockIdx.x == 0)         // an empty sequence has no tile to finish: it keeps nothing
+        for (int t = threadIdx.x; t < B * a.p.num_kv_heads; t += kThreadsTc)
+            if (a.seq_len[t / a.p.num_kv_heads] <= 0) a.sel_lengths[t] = 0;
     for (int t = threadIdx.x; t < B; t += kThreadsTc) t_start[t] = a.seq_start[t];
     if (threadIdx.x == 32) {
         int32_t pa = 0, ti = 0;
@@ -1055,7 +1116,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
     const int nitems = item1 - item0;
     if (warp < kEpiWarps) {
         EpiState es;
-        if (MODE == 4) epilogue_pass2(a, tl, sv, tmem_base, nitems, items, ctas, es);
+        if (MODE == 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, items, ctas, es);
         if (P1) epilogue_pass1(a, tl, tmem_base, nitems, es);
         if (MODE == 3) {
             // publish: this CTA's partials are in memory
@@ -1064,7 +1125,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
             if (threadIdx.x == 0)
                 asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(1u) : "memory");
         }
-        if (P2 && MODE != 4) epilogue_pass2(a, tl, sv, tmem_base, nitems, items, ctas, es);
+        if (P2 && MODE != 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, items, ctas, es);
     } else if (warp == kEpiWarps) {
         if (lane == 0) {
             RingState rs;
@@ -1074,6 +1135,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         }
     } else if (warp == kEpiWarps + 2) {
         if (a.cj.nslots > 0) copy_loop(a, tl, sv, smem_c, coff);
+    } else if (warp == kEpiWarps + 3) {
+        if (P2) finisher_pass2(a, tl, nitems, MODE == 3 ? (uint32_t)nitems : 0u);
     } else {
         if (lane == 0) {
             MmaState ms;
@@ -1125,7 +1188,7 @@ bool shape_for(const refree_params &p, TcShape &sh)
     sh.rblocks = (sh.R + kTile - 1) / kTile;
     sh.Rpad = sh.rblocks * kTile;
     sh.cblocks = sh.R > 256 ? 2 : 1;
-    sh.ncol = ((sh.R + sh.cblocks - 1) / sh.cblocks + 15) / 16 * 16;   // rows past R are masked by L = +inf
+    sh.ncol = ((sh.R + sh.cblocks - 1) / sh.cblocks + 31) / 32 * 32;   // two warps halve it in groups of 16; rows past R are masked
     sh.stages = sh.Rpad <= 256 ? 4 : 2;
     sh.rank4 = p.k_stride_seq != 0;
     return true;
@@ -1179,7 +1242,7 @@ cudaError_t device_info(DevInfo &out)
 bool copy_shape(const refree_params &p, TcShape &sh, int &nslots)
 {
     const int U = p.num_seqs * p.num_kv_heads;
-    if (sh.stages > 3) sh.stages = 3;
+    if (sh.stages > 2) sh.stages = 2;
     for (nslots = kMaxCopySlots; nslots >= 3; --nslots)
         if (smem_bytes(sh, p.num_seqs, nslots, U) <= kSmemLimit) return true;
     return false;
@@ -1266,6 +1329,9 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.scores = scores;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;
+    a.sel_lengths = nullptr;
+    a.sel_cuts = nullptr;
+    a.tickets = a.tickets_next = nullptr;
     a.cj = TcCopyJob{};
     const size_t smem = smem_bytes(sh, p.num_seqs);
     if (smem > kSmemLimit) return cudaErrorInvalidValue;
@@ -1297,7 +1363,8 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
 // stream, so no CTA waits for another and the launch is an ordinary one.
 cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, const TcLayer *finish,
                                  const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
-                                 const Workspace &lay, int32_t *dev_status, cudaStream_t st, const TcCopyJob *copy)
+                                 const Workspace &lay, int32_t *dev_status, cudaStream_t st, const TcCopyJob *copy,
+                                 bool finish_tickets_clean)
 {
     if (!begin && !finish) return cudaErrorInvalidValue;
     TcShape sh;
@@ -1328,6 +1395,17 @@ cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, c
     a.flags = nullptr;
     a.total_tokens = total_tokens;
     a.dev_status = dev_status;
+    // the rule runs inside the launch when the finished layer says where its budgets go
+    const bool sel = finish && finish->sel_lengths && finish->groups;
+    a.sel_lengths = sel ? finish->sel_lengths : nullptr;
+    a.sel_cuts = sel ? reinterpret_cast<Cut *>(finish->ws + lay.cut_off) : nullptr;
+    a.tickets = sel ? reinterpret_cast<uint32_t *>(finish->ws + lay.cnt_off) + kMaxCtas : nullptr;
+    a.tickets_next = (begin && begin->sel_lengths && begin->groups)
+                         ? reinterpret_cast<uint32_t *>(begin->ws + lay.cnt_off) + kMaxCtas : nullptr;
+    if (sel && !finish_tickets_clean) {
+        e = cudaMemsetAsync(a.tickets, 0, 2 * (size_t)p.num_seqs * p.num_kv_heads * sizeof(uint32_t), st);
+        if (e != cudaSuccess) return e;
+    }
     if (copy) a.cj = *copy; else a.cj = TcCopyJob{};
     a.cj.nslots = copy ? copy_slots : 0;
     const size_t smem = smem_bytes(sh, p.num_seqs, a.cj.nslots, p.num_seqs * p.num_kv_heads);

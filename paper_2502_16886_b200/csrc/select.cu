@@ -27,6 +27,7 @@
 #include <cooperative_groups.h>
 
 #include "refree_internal.cuh"
+#include "select_groups.cuh"
 
 namespace refree {
 namespace {
@@ -66,17 +67,6 @@ struct PosRank {     // position ranking: leading positions, then from the end b
 struct ProtRank {    // protected prefix of the score ranking: leading positions, then the window
     __device__ int operator()(const UnitView &v, int j) const { return j < v.lead ? j : v.n - v.w_eff + (j - v.lead); }
 };
-
-template <typename Tv> __device__ inline Tv warp_incl_scan(Tv x)
-{
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const Tv y = __shfl_up_sync(0xffffffffu, x, o);
-        if (lane >= o) x += y;
-    }
-    return x;
-}
 
 // Block-wide exclusive scan; `total` receives the sum.  `buf` holds kWarps + 1 items.
 template <typename Tv> __device__ inline Tv block_excl_scan(Tv x, Tv *buf, Tv &total)
@@ -266,16 +256,6 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
     const int S = 60 - ilogbf(fmaxf(acc, 0.25f)) - 2 * (emax - 127);
     v.sbias = S - 300;
     return true;
-}
-
-// Smallest fixed-point C with 1 - sqrt(C / Cn) < T, i.e. Cn - C < Cn * T * (2 - T); ~0 when there is none.
-__device__ inline u64 crossing_level(u64 Cn, double T)
-{
-    const double lim = (double)Cn * (T * (2.0 - T));
-    const double c = ceil(lim);
-    if (!(c >= 1.0)) return ~0ull;                 // T = 0: never met
-    const u64 dmax = (u64)c - 1ull;                // largest dropped mass that still meets the rule
-    return dmax >= Cn ? 0ull : Cn - dmax;
 }
 
 __global__ void __launch_bounds__(kThreads)

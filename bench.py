@@ -177,16 +177,25 @@ def algorithmic_bytes(cfg, seq_lens, lengths):
     return a, b4
 
 
-# dram__bytes_read + dram__bytes_write of one launch of the scoring kernel, from the ncu captures summarised
-# under profiles/: the 32K layer captured at full size; the 8K layer captured on the 8-layer cut of its workload.
-# Only for the kernel version the captures were taken on: window 64, tensor-core path.
-NCU_SCORE_TRAFFIC = {"llama3_8b_8k": 17_484_288, "mistral7b_32k": 68_277_504 + 2_643_200}
+# dram__bytes_read + dram__bytes_write of one launch of the dominant kernel, from the ncu capture summarised under
+# profiles/.  The figure belongs to one version of the kernel source: it is reported only while the source file
+# still has the hash it was captured on, and null afterwards.
+NCU_TRAFFIC = {
+    # workload: (kernel source, first 16 hex digits of its sha256, bytes per launch)
+}
 
 
 def ncu_traffic(cfg, stage):
-    if stage != "score" or cfg.window != 64:
+    import hashlib
+    rec = NCU_TRAFFIC.get(cfg.name)
+    if stage != "score" or cfg.window != 64 or rec is None:
         return None
-    return NCU_SCORE_TRAFFIC.get(cfg.name)
+    src, digest, nbytes = rec
+    try:
+        have = hashlib.sha256(open(os.path.join(ROOT, src), "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return nbytes if have == digest else None
 
 
 def run_ours(args):
@@ -215,7 +224,7 @@ def run_ours(args):
     for l in range(L):
         lay = workloads.make_layer(cfg, l)
         if params is None:
-            params = binding.params_for(cfg, lay, rank_mode=rank_mode)
+            params = binding.params_for(cfg, lay, rank_mode=rank_mode, threshold=args.threshold)
         layers.append(dict(
             q=lay.q_win.to(dev), k=lay.k.to(dev), v=lay.v.to(dev),
             k_out=torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype, device=dev),
@@ -273,10 +282,18 @@ def run_ours(args):
         time.sleep(0.3)
     launches0 = binding.refree_kernel_launch_count()
     sampler.mark_begin()
-    ms_local = timed(step, args.steps)
+    # blocks of exactly `steps` steps, each bracketed by barrier + synchronize and timed with CUDA events; repeated
+    # until a second of device time has gone by (so the clock sampler sees the load), the median block is reported
+    block_ms, spent = [], 0.0
+    while not block_ms or (spent < 1000.0 and len(block_ms) < 64):
+        block_ms.append(timed(step, args.steps))
+        spent += block_ms[-1] * args.steps
+        if world > 1:
+            spent = dist_max(spent, world, dev)      # every rank runs the same number of blocks
+    ms_local = statistics.median(block_ms)
     sampler.mark_end()
     dist_barrier(world)
-    launches = binding.refree_kernel_launch_count() - launches0
+    launches = (binding.refree_kernel_launch_count() - launches0) // len(block_ms)
     clocks = sampler.stop() if rank == 0 else None
     ms_step = dist_max(ms_local, world, dev)
     ms_per_layer_calls = dist_max(ms_per_layer_calls, world, dev)
@@ -452,22 +469,86 @@ def run_ours(args):
     else:
         inplace_line = None
 
+    # the same step in the paper's other settings, on the same device-resident cache: ranking by score (Section 4.4)
+    # and the default single query row (Section 3.2 "Reducing Overhead"; the window's last row of every head)
+    def variant_record(p_var, qs):
+        pv = binding.LayerPointers(qs, *[[d[key] for d in layers] for key in ("k", "v", "k_out", "v_out", "lengths", "offsets")])
+        wsv = torch.empty(binding.refree_layers_workspace_size(p_var, total), dtype=torch.uint8, device=dev)
+
+        def run():
+            binding.refree_compress_layers(p_var, pv, seq_start, seq_len, total, cap, wsv, status)
+        for _ in range(3):
+            run()
+        ms = statistics.median(timed(run, 5) for _ in range(3)) / L
+        assert int(status.item()) == 0, f"device status {int(status.item())}"
+        ln = [d["lengths"].view(len(seq_lens), cfg.num_kv_heads).cpu().tolist() for d in layers]
+        b3 = sum(algorithmic_bytes(cfg, seq_lens, x)[0] for x in ln) / L
+        r = sum(sum(map(sum, x)) for x in ln) / (L * cfg.num_kv_heads * total)
+        return {"us_per_layer": round(ms * 1e3, 2), "tokens_per_s_per_layer": round(total / (ms * 1e-3), 1),
+                "kept_ratio": round(r, 4), "achieved": round(b3 / (ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "frac": round(b3 / (ms * 1e-3) / 1e9 / peak, 4), "peak_kind": f"of {peak_kind}"}
+
+    import dataclasses as _dc
+    sub = {}
+    if not args.no_variants and world == 1:
+        other = binding.RANK_POSITION if rank_mode == binding.RANK_SCORE else binding.RANK_SCORE
+        p_other = _dc.replace(params, rank_mode=other)
+        sub["score_mode" if other == binding.RANK_SCORE else "position_mode"] = variant_record(p_other, [d["q"] for d in layers])
+        if cfg.window > 1:
+            p_w1 = _dc.replace(params, window=1)
+            sub["window_1"] = variant_record(p_w1, [d["q"][:, :, -1:, :].contiguous() for d in layers])
+        step()                                   # leave the headline setting's budgets behind for what follows
+        torch.cuda.synchronize()
+
+    # what traffic of this shape can reach on the device: a read-only stream over one layer's K, and a row copy that
+    # reads (1 + rho) and writes 2 rho of a layer's bytes, each swept over the layers like a stage
+    def sweep_ms(call):
+        for d in layers:
+            call(d)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for d in layers:
+                call(d)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * L)
+
+    rows_all = cfg.num_kv_heads * total
+    kept_all = int(round(rho * rows_all))
+    ceiling = {"rho": round(rho, 4),
+               "how": "hand-written probes of the library: refree_sol_read_stream over a layer's K; refree_sol_row_mix "
+                      "reads (1 + rho) and writes 2 rho of a layer's K/V bytes in 256-byte rows; swept over the layers; "
+                      "each with vector loads/stores in registers and with the bulk-copy engine"}
+    for tag, bulk in (("ldst", False), ("bulk", True)):
+        read_ms = sweep_ms(lambda d: binding.refree_sol_read_stream(d["k"], bulk=bulk))
+        mix_ms = sweep_ms(lambda d: binding.refree_sol_row_mix(d["k"], d["v"], d["k_out"], d["v_out"], rows_all, kept_all,
+                                                               row, bulk=bulk))
+        ceiling[f"read_stream_{tag}_gbs"] = round(rows_all * row / (read_ms * 1e-3) / 1e9, 1)
+        ceiling[f"row_mix_{tag}_gbs"] = round((rows_all + 3 * kept_all) * row / (mix_ms * 1e-3) / 1e9, 1)
+    ceiling["row_mix_gbs"] = max(ceiling["row_mix_ldst_gbs"], ceiling["row_mix_bulk_gbs"])
+    step()                                       # the probes overwrote the outputs: put the pass's results back
+    torch.cuda.synchronize()
+
     e2e = measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args)
     cpu_baseline = measure_cpu_baseline(cfg, rank_mode, total, args) if world == 1 and not args.no_cpu_baseline else None
 
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": True,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "blocks_timed": len(block_ms),
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.num_q_heads, "kv_heads": cfg.num_kv_heads,
                    "head_dim": cfg.head_dim, "seq_lens": seq_lens if len(seq_lens) <= 8 else len(seq_lens),
-                   "window": cfg.window, "sink": cfg.sink, "threshold": 0.01, "rank_mode": args.rank_mode,
+                   "window": cfg.window, "sink": cfg.sink, "threshold": args.threshold, "rank_mode": args.rank_mode,
                    "scope": "head", "layout": "head_major",
                    "l2": f"each step sweeps {L} layers of distinct K/V buffers "
                          f"({L * 2 * cfg.num_kv_heads * total * row / 2**30:.1f} GiB), larger than L2",
                    "replicas": world},
         "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
-        "roofline": roofline, "roofline_pass": roofline_pass, "decode_attention": decode_line,
+        "roofline": roofline, "roofline_pass": roofline_pass, "ceiling_gbs": ceiling["row_mix_gbs"], "ceiling": ceiling,
+        **sub, "decode_attention": decode_line,
         "compact_inplace": inplace_line,
         "cpu_baseline": cpu_baseline,
     }
@@ -536,7 +617,7 @@ def measure_e2e(binding, workloads, cfg, params, dev, L, total, cap, units, args
 
 
 # --------------------------------------------------------- CPU oracle arm ----
-def oracle_sample(cfg, rank_mode, layer_idx, heads):
+def oracle_sample(cfg, rank_mode, layer_idx, heads, threshold=0.01):
     """Inputs of the oracle for `heads` KV heads of one layer of the workload."""
     from oracle import refree_oracle as orc
     from paper_2502_16886_b200 import workloads
@@ -544,7 +625,7 @@ def oracle_sample(cfg, rank_mode, layer_idx, heads):
     G = cfg.group
     total = lay.total_tokens
     p = orc.OracleParams(int(lay.seq_len.numel()), heads * G, heads, cfg.head_dim, window=cfg.window, sink=cfg.sink,
-                         rank_mode=rank_mode, dtype=0 if cfg.dtype == "fp32" else 1,
+                         threshold=threshold, rank_mode=rank_mode, dtype=0 if cfg.dtype == "fp32" else 1,
                          k_strides=(0, cfg.head_dim, total * cfg.head_dim),
                          v_strides=(0, cfg.head_dim, total * cfg.head_dim))
     return p, lay.q_win[:, :heads * G].contiguous(), lay.k[:heads].contiguous(), lay.v[:heads].contiguous(), \
@@ -565,16 +646,32 @@ def measure_cpu_baseline(cfg, rank_mode, total, args):
     heads = oracle_heads_for_budget(cfg, total)
     t_used, n_calls, layer = 0.0, 0, 0
     while t_used < 10.0 and n_calls < 8:
-        inp = oracle_sample(cfg, rank_mode, layer % cfg.num_layers, heads)
+        inp = oracle_sample(cfg, rank_mode, layer % cfg.num_layers, heads, args.threshold)
         t0 = time.perf_counter()
         orc.compress_layer(*inp)
         t_used += time.perf_counter() - t0
         n_calls += 1
         layer += 1
     per_layer = t_used / n_calls * cfg.num_kv_heads / heads
-    return {"value": round(total / per_layer, 1), "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
-            "sample": f"{n_calls} layer(s) of {cfg.name}, {heads} of {cfg.num_kv_heads} KV heads each, "
-                      f"scaled to a full layer; {t_used:.1f}s of CPU time"}
+    out = {"value": round(total / per_layer, 1), "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+           "sample": f"{n_calls} layer(s) of {cfg.name}, {heads} of {cfg.num_kv_heads} KV heads each, "
+                     f"scaled to a full layer; {t_used:.1f}s of CPU time"}
+    # one thread, on the 8K-token Llama3-8B-shaped cache: one KV head of one layer, scaled to the layer
+    from paper_2502_16886_b200 import workloads
+    cfg8 = workloads.get_config("llama3_8b_8k")
+    threads = orc.num_threads()
+    try:
+        orc.set_num_threads(1)
+        inp = oracle_sample(cfg8, rank_mode, 0, 1)
+        t0 = time.perf_counter()
+        orc.compress_layer(*inp)
+        dt = time.perf_counter() - t0
+    finally:
+        orc.set_num_threads(threads)
+    tot8 = sum(workloads.sequence_lengths(cfg8))
+    out["single_thread_llama3_8b_8k"] = {"value": round(tot8 / (dt * cfg8.num_kv_heads), 1), "unit": UNIT, "cores": 1,
+                                         "sample": f"1 of {cfg8.num_kv_heads} KV heads of one layer, scaled; {dt:.1f}s"}
+    return out
 
 
 def run_reference(args):
@@ -589,7 +686,7 @@ def run_reference(args):
     seq_lens = workloads.sequence_lengths(cfg)
     total = sum(seq_lens)
     heads = oracle_heads_for_budget(cfg, total, seconds=2.0)
-    samples = [oracle_sample(cfg, rank_mode, l, heads) for l in range(min(2, cfg.num_layers))]
+    samples = [oracle_sample(cfg, rank_mode, l, heads, args.threshold) for l in range(min(2, cfg.num_layers))]
     for i in range(args.warmup):
         orc.compress_layer(*samples[i % len(samples)])
     t0 = time.perf_counter()
@@ -598,16 +695,86 @@ def run_reference(args):
     dt = (time.perf_counter() - t0) / args.steps
     per_layer = dt * cfg.num_kv_heads / heads
     value = round(total / per_layer, 1)
-    sample = (f"one step = one layer of {cfg.name}, {heads} of {cfg.num_kv_heads} KV heads, "
-              f"scaled to a full layer; host-resident inputs")
+    sample = (f"one step = {heads} of {cfg.num_kv_heads} KV heads of one layer of {cfg.name} (a bounded sample of the "
+              f"workload); value = tokens / (step time x {cfg.num_kv_heads}/{heads}); host-resident inputs")
+    row = cfg.head_dim * cfg.elem_bytes
+    L = cfg.num_layers
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(per_layer * cfg.num_layers * 1e3, 3),
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3),
+            "scaled_to_full_layer": {"ms_per_layer": round(per_layer * 1e3, 3), "kv_heads_timed": heads,
+                                     "kv_heads": cfg.num_kv_heads},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "layers": cfg.num_layers, "rank_mode": args.rank_mode, "window": cfg.window},
+            "config": {"workload": cfg.name, "layers": L, "q_heads": cfg.num_q_heads, "kv_heads": cfg.num_kv_heads,
+                       "head_dim": cfg.head_dim, "seq_lens": seq_lens if len(seq_lens) <= 8 else len(seq_lens),
+                       "window": cfg.window, "sink": cfg.sink, "threshold": args.threshold, "rank_mode": args.rank_mode,
+                       "scope": "head", "layout": "head_major",
+                       "l2": f"each step sweeps {L} layers of distinct K/V buffers "
+                             f"({L * 2 * cfg.num_kv_heads * total * row / 2**30:.1f} GiB), larger than L2",
+                       "replicas": world},
             "gpu_launches": 0,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+def run_sweep(args):
+    """The paper's ablations as a second workload (Section 4.4: the window k as a share of n; Section 3.2: T between
+    0.1 % and 10 %): one refree_compress_layers call over a cut of the 8K cache per point.  A window whose row count
+    the library does not take is reported as unsupported, not skipped."""
+    from paper_2502_16886_b200 import binding, build, workloads
+    import dataclasses
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", 0)
+    build.build()
+    binding.lib()
+    base = workloads.get_config("llama3_8b_8k")
+    L = args.layers or 8
+    n = workloads.sequence_lengths(base)[0]
+    points = []
+    for window in (1, max(1, round(0.01 * n)), round(0.05 * n), round(0.10 * n)):
+        cfg = dataclasses.replace(base, window=window)
+        rows = cfg.group * window
+        if rows > 1024:
+            points += [{"window": window, "threshold": t, "status": "unsupported: G * window = %d rows > 1024" % rows}
+                       for t in (0.001, 0.01, 0.1)]
+            continue
+        lays = [workloads.make_layer(cfg, l) for l in range(L)]
+        total = lays[0].total_tokens
+        cap = cfg.num_kv_heads * total
+        units = cfg.num_kv_heads
+        dv = [dict(q=x.q_win.to(dev), k=x.k.to(dev), v=x.v.to(dev),
+                   k_out=torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype, device=dev),
+                   v_out=torch.empty(cap, cfg.head_dim, dtype=cfg.torch_dtype, device=dev),
+                   lengths=torch.zeros(units, dtype=torch.int32, device=dev),
+                   offsets=torch.zeros(units + 1, dtype=torch.int64, device=dev)) for x in lays]
+        ss, sl = lays[0].seq_start.to(dev), lays[0].seq_len.to(dev)
+        ptrs = binding.LayerPointers(*[[d[key] for d in dv] for key in ("q", "k", "v", "k_out", "v_out", "lengths", "offsets")])
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        for t in (0.001, 0.01, 0.1):
+            p = binding.params_for(cfg, lays[0], threshold=t)
+            ws = torch.empty(binding.refree_layers_workspace_size(p, total), dtype=torch.uint8, device=dev)
+
+            def run():
+                binding.refree_compress_layers(p, ptrs, ss, sl, total, cap, ws, status)
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            ms = e0.elapsed_time(e1) / (10 * L)
+            rho = sum(int(d["lengths"].sum()) for d in dv) / (L * cap)
+            points.append({"window": window, "threshold": t, "us_per_layer": round(ms * 1e3, 2),
+                           "tokens_per_s_per_layer": round(total / (ms * 1e-3), 1), "kept_ratio": round(rho, 4)})
+        del dv, lays
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": "threshold x window on llama3_8b_8k (Section 4.4, Section 3.2)",
+                      "layers": L, "rank_mode": "position", "data": "synthetic", "points": points}), flush=True)
 
 
 def main():
@@ -621,9 +788,16 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debugging: use fewer layers than the config")
     ap.add_argument("--window", type=int, default=0, help="override the config's observation window (paper default: 1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the score-ranking and single-row sub-records")
+    ap.add_argument("--threshold", type=float, default=0.01, help="the stopping rule's T (paper: 1 %%)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="second workload: T in {0.1 %%, 1 %%, 10 %%} x window in {1, 1 %%n, 5 %%n, 10 %%n} on the 8K cache")
     ap.add_argument("--per-layer-calls", action="store_true",
                     help="time one refree_compress_layer call per layer instead of one refree_compress_layers call per step")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 5
         args.warmup = args.warmup if args.warmup is not None else 1

@@ -380,6 +380,26 @@ refree_status refree_decode_attention_inplace(const refree_params *params, const
  * library has enqueued in this process so far (all entry points, all streams). */
 int64_t refree_kernel_launch_count(void);
 
+/* Measurement aids with no counterpart in the paper: two memory-system probes with the
+ * access shape of the pass (Section 3.2's O(n) claim is a statement about exactly this
+ * traffic), used by the benchmark to report what such traffic can reach on the device.
+ *   refree_sol_read_stream  reads `bytes` (a multiple of 16) from src (device, 16-byte
+ *                           aligned) once: the K stream of scoring.
+ *   refree_sol_row_mix      reads rows [0, rows) of k, and copies the last kept_rows rows
+ *                           of k and of v to k_out and v_out: (rows + kept_rows) rows
+ *                           read, 2 * kept_rows written, the mix of the whole pass.
+ * `sink` (device int32, nullable) only keeps the loads alive; nothing meaningful is
+ * written to it.  Passing REFREE_SOL_BULK as `sink` selects the variant that moves the same
+ * bytes with the bulk-copy engine (global -> shared -> global in 16 KB pieces) instead of
+ * vector loads and stores in registers; its first call on a device sets a kernel attribute
+ * and should come before any stream capture.  Errors: REFREE_ERR_INVALID_ARG for null, misaligned or negative
+ * arguments; nothing is launched then. */
+#define REFREE_SOL_BULK ((int32_t *)(uintptr_t)1)
+refree_status refree_sol_read_stream(const void *src, int64_t bytes, int32_t *sink, void *stream);
+refree_status refree_sol_row_mix(const void *k, const void *v, void *k_out, void *v_out,
+                                 int64_t rows, int64_t kept_rows, int32_t row_bytes,
+                                 int32_t *sink, void *stream);
+
 /* Static string for a status code. */
 const char *refree_status_string(refree_status s);
 

@@ -105,6 +105,8 @@ SIGNATURES = {
     "refree_decode_attention": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _I64, _VP, _VP, _SZ, _VP, _VP]),
     "refree_decode_attention_inplace": (ctypes.c_int, [_PP, _VP, _VP, _VP, _VP, _VP, _VP, ctypes.c_int32, _I64, _VP, _VP,
                                                        _SZ, _VP, _VP]),
+    "refree_sol_read_stream": (ctypes.c_int, [_VP, _I64, _VP, _VP]),
+    "refree_sol_row_mix": (ctypes.c_int, [_VP, _VP, _VP, _VP, _I64, _I64, ctypes.c_int32, _VP, _VP]),
     "refree_host_arena_size": (ctypes.c_int, [_PP, _I64, _I64, _I64, ctypes.POINTER(_SZ)]),
     "refree_compress_layer_host": (ctypes.c_int, [_PP, _VP, _VP, _VP, _I64, _VP, _VP, _I64, _VP, _VP, _I64,
                                                   _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
@@ -342,6 +344,19 @@ def refree_compress_layers_host(p: Params, q_win, k, v, seq_start, seq_len, tota
     if check:
         _check(rc, "refree_compress_layers_host")
     return rc
+
+
+def refree_sol_read_stream(src: torch.Tensor, stream=None, bulk=False) -> None:
+    """Read every byte of ``src`` once (memory-system probe; ``bulk``: through the bulk-copy engine)."""
+    _check(lib().refree_sol_read_stream(_dp(src), ctypes.c_int64(src.numel() * src.element_size()),
+                                        ctypes.c_void_p(1) if bulk else None, _stream(stream)), "refree_sol_read_stream")
+
+
+def refree_sol_row_mix(k, v, k_out, v_out, rows: int, kept_rows: int, row_bytes: int, stream=None, bulk=False) -> None:
+    """Read ``rows`` rows of ``k``; copy the last ``kept_rows`` rows of ``k`` and ``v`` (memory-system probe)."""
+    _check(lib().refree_sol_row_mix(_dp(k), _dp(v), _dp(k_out), _dp(v_out), ctypes.c_int64(rows), ctypes.c_int64(kept_rows),
+                                    ctypes.c_int32(row_bytes), ctypes.c_void_p(1) if bulk else None, _stream(stream)),
+           "refree_sol_row_mix")
 
 
 def refree_layers_workspace_size(p: Params, total_tokens: int) -> int:

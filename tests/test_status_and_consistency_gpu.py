@@ -98,3 +98,18 @@ def test_fused_budgets_equal_the_staged_selection_on_the_same_gpu_scores(name):
     np.testing.assert_array_equal(lengths.cpu().numpy(), res.lengths.reshape(-1).cpu().numpy())
     np.testing.assert_array_equal(offsets.cpu().numpy(), res.offsets.cpu().numpy())
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("bulk", [False, True])
+def test_memory_probes_copy_the_rows_they_say(bulk):
+    # the probes only exist to put a ceiling beside the benchmark's numbers, but what they move must be right
+    rows, kept, d = 5000, 4321, 128
+    k = torch.randn(rows, d, device=DEV).to(torch.bfloat16)
+    v = torch.randn(rows, d, device=DEV).to(torch.bfloat16)
+    k_out = torch.zeros(kept, d, dtype=torch.bfloat16, device=DEV)
+    v_out = torch.zeros(kept, d, dtype=torch.bfloat16, device=DEV)
+    binding.refree_sol_row_mix(k, v, k_out, v_out, rows, kept, d * 2, bulk=bulk)
+    binding.refree_sol_read_stream(k, bulk=bulk)
+    torch.cuda.synchronize()
+    assert torch.equal(parity.bits(k_out), parity.bits(k[rows - kept:]))
+    assert torch.equal(parity.bits(v_out), parity.bits(v[rows - kept:]))

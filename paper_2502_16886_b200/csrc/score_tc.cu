@@ -332,7 +332,7 @@ struct EpiState { uint32_t ephase = 0, icount = 0; };
 // --------------------------------------------------------- producer / MMA -----
 __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, const CUtensorMap *mapk,
                                      unsigned char *smem_q, unsigned char *smem_k, TcSmemTail &tl, const SeqView &sv,
-                                     int item0, int item1, RingState &rs)
+                                     int item0, int item1, RingState &rs, bool reverse)
 {
     const TcShape &sh = a.sh;
     const int G = a.p.num_q_heads / a.p.num_kv_heads, Hkv = a.p.num_kv_heads;
@@ -340,9 +340,15 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     int &stage = rs.stage;
     uint32_t &kphase = rs.kphase, &qphase = rs.qphase;
     bool ok = true;
+    // The column pass walks its items backwards: the row pass before it (of the same layer, in this launch or at
+    // the end of the launch before) left its last K tiles in L2, and those are asked for first.
     ItemTc it = {};
-    if (item0 < item1) it = decode_item_tc(sv, a.p.num_seqs, Hkv, item0);
-    for (int item = item0; item < item1 && ok; ++item, next_item_tc(it, sv, a.p.num_seqs, Hkv)) {
+    if (item0 < item1) it = decode_item_tc(sv, a.p.num_seqs, Hkv, reverse ? item1 - 1 : item0);
+    for (int x = 0; x < item1 - item0 && ok; ++x) {
+        if (x > 0) {
+            if (reverse) it = decode_item_tc(sv, a.p.num_seqs, Hkv, item1 - 1 - x);
+            else next_item_tc(it, sv, a.p.num_seqs, Hkv);
+        }
         const bool new_unit = it.u != cur_u;
         // the ring entry was last used sixteen items ago, which every consumer has long left behind
         ItemInfo &inf = tl.info[rs.icount++ & (kInfoRing - 1)];
@@ -790,17 +796,17 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
     bool ok = true;
     for (int item = 0; item < nitems && ok; ++item) {
         const ItemInfo *inf = &tl.info[es.icount++ & (kInfoRing - 1)];
-        if (item == next_change) {
+        if (item == next_change) {   // `item` counts the pass's items in the order they come: from the CTA's last one backwards
             // A unit begins: all sixteen warps meet (the two groups share L), whichever group takes the item's
             // products.  The unit is looked up in the sequence tables, not in the item's record, which a warp
             // that takes none of the item's products has no barrier to wait for.  The normalisers do not wait
             // for the tile either: the partials come from the row pass, not from anything this pass loads.
-            const ItemTc it = decode_item_tc(sv, a.p.num_seqs, a.p.num_kv_heads, item0 + item);
+            const ItemTc it = decode_item_tc(sv, a.p.num_seqs, a.p.num_kv_heads, item0 + (nitems - 1 - item));
             if (item > 0 && !(ok = epi_sync(tl, ephase))) break;   // nobody still reads the previous unit's L
             ok = merge_unit_lse(a, tl, it.u, sv.tiles[it.s] * a.p.num_kv_heads + it.g * it.ntiles, it.ntiles, items, ctas,
                                 ephase);
             if (!ok) break;
-            next_change = item + (it.ntiles - it.tile);
+            next_change = item + it.tile + 1;                      // the unit's earlier tiles follow
         }
         for (int cb = 0; cb < sh.cblocks && ok; ++cb) {
             const uint32_t j = (uint32_t)item * (uint32_t)sh.cblocks + (uint32_t)cb;      // product index in this pass
@@ -1129,9 +1135,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
     } else if (warp == kEpiWarps) {
         if (lane == 0) {
             RingState rs;
-            if (MODE == 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs);
-            if (P1) producer_loop(a, &mapq_a, &mapk_a, smem_q, smem_k, tl, sv, item0, item1, rs);
-            if (P2 && MODE != 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs);
+            if (MODE == 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs, true);
+            if (P1) producer_loop(a, &mapq_a, &mapk_a, smem_q, smem_k, tl, sv, item0, item1, rs, false);
+            if (P2 && MODE != 4) producer_loop(a, &mapq_b, &mapk_b, smem_q, smem_k, tl, sv, item0, item1, rs, true);
         }
     } else if (warp == kEpiWarps + 2) {
         if (a.cj.nslots > 0) copy_loop(a, tl, sv, smem_c, coff);

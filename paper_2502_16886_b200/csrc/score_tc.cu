@@ -309,6 +309,7 @@ struct TcArgs {
     Cut *sel_cuts;             // [units]
     uint32_t *tickets;         // [2 units] tiles finished per unit, then the unit's largest score; zero when the launch begins
     uint32_t *tickets_next;    // [2 units] those of the launch that follows, cleared by this one
+    int dependent;             // launched with programmatic stream serialization: wait for the launch before
     TcCopyJob cj;          // rows of an earlier layer to move while this layer is scored (nslots == 0: none)
 };
 
@@ -1085,11 +1086,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         tl.abort_flag = 0;
         fence_barrier_init();
     }
-    if (a.tickets_next && blockIdx.x == 0)
-        for (int t = threadIdx.x; t < 2 * B * a.p.num_kv_heads; t += kThreadsTc) a.tickets_next[t] = 0u;
-    if (a.sel_lengths && blockIdx.x == 0)         // an empty sequence has no tile to finish: it keeps nothing
-        for (int t = threadIdx.x; t < B * a.p.num_kv_heads; t += kThreadsTc)
-            if (a.seq_len[t / a.p.num_kv_heads] <= 0) a.sel_lengths[t] = 0;
     for (int t = threadIdx.x; t < B; t += kThreadsTc) t_start[t] = a.seq_start[t];
     if (threadIdx.x == 32) {
         int32_t pa = 0, ti = 0;
@@ -1109,6 +1105,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tl.tmem_base;
+    // Everything up to here is local to the CTA or reads the caller's inputs.  In a run of layers the launch may have been started while the
+    // launch before it was still draining (programmatic dependent launch): from here on its results are needed.
+    if (a.dependent) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (a.tickets_next && blockIdx.x == 0)
+        for (int t = threadIdx.x; t < 2 * B * a.p.num_kv_heads; t += kThreadsTc) a.tickets_next[t] = 0u;
+    if (a.sel_lengths && blockIdx.x == 0)         // an empty sequence has no tile to finish: it keeps nothing
+        for (int t = threadIdx.x; t < B * a.p.num_kv_heads; t += kThreadsTc)
+            if (a.seq_len[t / a.p.num_kv_heads] <= 0) a.sel_lengths[t] = 0;
     SeqView sv;
     sv.pack = t_pack; sv.tiles = t_tiles; sv.len = t_len; sv.start = t_start;
 
@@ -1338,6 +1342,7 @@ cudaError_t launch_score_tc(const refree_params &p, const void *q_win, const voi
     a.sel_lengths = nullptr;
     a.sel_cuts = nullptr;
     a.tickets = a.tickets_next = nullptr;
+    a.dependent = 0;
     a.cj = TcCopyJob{};
     const size_t smem = smem_bytes(sh, p.num_seqs);
     if (smem > kSmemLimit) return cudaErrorInvalidValue;
@@ -1416,9 +1421,23 @@ cudaError_t launch_score_tc_pipe(const refree_params &p, const TcLayer *begin, c
     a.cj.nslots = copy ? copy_slots : 0;
     const size_t smem = smem_bytes(sh, p.num_seqs, a.cj.nslots, p.num_seqs * p.num_kv_heads);
     if (smem > kSmemLimit) return cudaErrorInvalidValue;
-    if (begin && finish) score_tc_kernel<4><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
-    else if (begin) score_tc_kernel<1><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
-    else score_tc_kernel<2><<<ctas, kThreadsTc, smem, st>>>(mapq_a, mapk_a, mapq_b, mapk_b, a);
+    // Launches of a run after the first may start while the one before drains: their CTAs set themselves up and
+    // then wait (griddepcontrol.wait) until that launch has completed and its results are visible.
+    a.dependent = finish_tickets_clean ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.dependent ? 1 : 0;
+    if (begin && finish) e = cudaLaunchKernelEx(&cfg, score_tc_kernel<4>, mapq_a, mapk_a, mapq_b, mapk_b, a);
+    else if (begin) e = cudaLaunchKernelEx(&cfg, score_tc_kernel<1>, mapq_a, mapk_a, mapq_b, mapk_b, a);
+    else e = cudaLaunchKernelEx(&cfg, score_tc_kernel<2>, mapq_a, mapk_a, mapq_b, mapk_b, a);
+    if (e != cudaSuccess) return e;
     count_launches(1);
     return cudaGetLastError();
 }

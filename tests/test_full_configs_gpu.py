@@ -26,7 +26,12 @@ def test_full_size_layer_matches_oracle(name, layer, rank_mode):
     lay = workloads.make_layer(cfg, layer)
     res, ref, worst, ties = parity.run_fused_and_check(cfg, lay, rank_mode=rank_mode)
     units = res.lengths.numel()
-    assert ties <= max(1, units // 4), f"{ties} of {units} units needed the near-tie rule"
+    print(f"{name} layer {layer} rank_mode {rank_mode}: {ties} of {units} units under the near-tie rule, "
+          f"worst score error {worst:.2e} relative")
+    # observed on every config and both rankings: no unit needs the near-tie rule (budgets and kept sets equal the
+    # oracle's outright), and the scores agree to 1e-6; a regression in either shows here, not behind a loose bound
+    assert ties == 0, f"{ties} of {units} units needed the near-tie rule"
+    assert worst < 1e-5
     rho = float(res.lengths.sum()) / (cfg.num_kv_heads * lay.total_tokens)
     assert 0.0 < rho <= 1.0
     torch.cuda.empty_cache()
@@ -70,9 +75,9 @@ def test_decode_attention_over_the_compacted_layer_at_full_size(name):
 @pytest.mark.parametrize("name,n_layers", [("mistral7b_32k", 4), ("qwen25_7b_ragged8", 3)])
 def test_one_call_run_of_layers_at_full_size(name, n_layers):
     """The step the benchmark times: refree_compress_layers over consecutive full-size layers (both
-    workspace halves reused).  Budgets and every compacted row against the oracle; a layer whose budgets
-    differ from the oracle's (near-ties, judged by the per-layer test above) is compared with the
-    per-layer call instead, which must agree with the one-call run bit for bit in any case."""
+    workspace halves reused).  Budgets and every compacted row against the oracle (every layer's budgets equal
+    the oracle's on these workloads), and against the per-layer call, which must agree with the one-call run
+    bit for bit in any case."""
     from oracle import refree_oracle as orc
     cfg = workloads.get_config(name)
     dev = "cuda:0"
@@ -110,5 +115,5 @@ def test_one_call_run_of_layers_at_full_size(name, n_layers):
             assert torch.equal(parity.bits(k_out[l][:rows].cpu()), parity.bits(ref.k_out))
             assert torch.equal(parity.bits(v_out[l][:rows].cpu()), parity.bits(ref.v_out))
         del one
-    assert exact >= n_layers - 1, f"only {exact} of {n_layers} layers had the oracle's budgets exactly"
+    assert exact == n_layers, f"only {exact} of {n_layers} layers had the oracle's budgets exactly"
     torch.cuda.empty_cache()

@@ -103,15 +103,17 @@ __device__ inline void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
 }
-__device__ inline void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
+// K tiles carry an L2 eviction priority: the row pass reads a tile first (keep it: the column pass comes back for
+// it), the column pass reads it last (let it go first).
+__device__ inline void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, uint64_t pol)
 {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
 }
-__device__ inline void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3)
+__device__ inline void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3, uint64_t pol)
 {
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
 }
 
 __device__ inline void tmem_alloc(uint32_t *dst_smem, uint32_t cols)
@@ -343,6 +345,9 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
     bool ok = true;
     // The column pass walks its items backwards: the row pass before it (of the same layer, in this launch or at
     // the end of the launch before) left its last K tiles in L2, and those are asked for first.
+    uint64_t pol;
+    if (reverse) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
     ItemTc it = {};
     if (item0 < item1) it = decode_item_tc(sv, a.p.num_seqs, Hkv, reverse ? item1 - 1 : item0);
     for (int x = 0; x < item1 - item0 && ok; ++x) {
@@ -364,9 +369,9 @@ __device__ inline void producer_loop(const TcArgs &a, const CUtensorMap *mapq, c
         unsigned char *dst = smem_k + (size_t)stage * kTileBytes;
         for (int h = 0; h < 2; ++h) {
             if (sh.rank4)
-                tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s);
+                tma_load_4d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, it.s, pol);
             else
-                tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g);
+                tma_load_3d(dst + h * kHalfBytes, mapk, &tl.k_full[stage], h * 64, it.tok0 + it.tile_start, it.g, pol);
         }
         if (new_unit) {
             ok = mbar_wait(&tl.q_empty, qphase ^ 1, &tl.abort_flag);
@@ -967,9 +972,8 @@ __device__ inline void copy_loop(const TcArgs &a, TcSmemTail &tl, const SeqView 
     const int nslots = cj.nslots;
     if (lane >= nslots || rows <= 0) return;
 
-    // Lane j owns slot j and every nslots-th piece of this CTA; the lanes move in step: all load, all wait,
-    // all store, all wait until their stores have read the slots.
-    const unsigned workers = (1u << nslots) - 1u;
+    // Lane j owns slot j and every nslots-th piece of this CTA, and runs its own load -> wait -> store -> wait
+    // chain; the lanes drift apart, which spreads the requests in time.
     const int64_t k_tok = a.p.k_stride_tok * 2, v_tok = a.p.v_stride_tok * 2;      // bytes (bf16)
     const int64_t pieces_per_array = (rows + kCopyRows - 1) / kCopyRows, pieces = 2 * pieces_per_array;
     int64_t next = blockIdx.x + (int64_t)lane * gridDim.x;      // next piece of this lane
@@ -1002,7 +1006,7 @@ __device__ inline void copy_loop(const TcArgs &a, TcSmemTail &tl, const SeqView 
                 u_cur = lo;
             }
         }
-        if (!__any_sync(workers, has)) break;
+        if (!has) break;
         unsigned char *dst = nullptr;
         uint32_t bytes = 0;
         if (has) {
@@ -1033,7 +1037,7 @@ __device__ inline void copy_loop(const TcArgs &a, TcSmemTail &tl, const SeqView 
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             }
         }
-        ok = !__any_sync(workers, !ok) && !tl.abort_flag;
+        ok = ok && !tl.abort_flag;
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }

@@ -235,9 +235,10 @@ struct TcSmemTail {
 };
 
 // Per-sequence tables of the CTA behind the tail, sized by the number of sequences:
-// pack[B + 1], tiles[B + 1] (running sums of lengths and of tiles), len[B], start[B].
+// pack[B + 1], tiles[B + 1] (running sums of lengths and of tiles), len[B], start[B], ne[B + 1] (non-empty
+// sequences before each).
 struct SeqView {
-    const int32_t *pack, *tiles, *len, *start;
+    const int32_t *pack, *tiles, *len, *start, *ne;
 };
 
 struct ItemTc {
@@ -289,8 +290,55 @@ __device__ inline void next_item_tc(ItemTc &it, const SeqView &sv, int B, int Hk
     fill_seq_fields(it, sv, Hkv);
 }
 
-// first item of CTA c when `items` are split evenly over `ctas`
-__device__ __host__ inline int range_begin(int c, int items, int ctas) { return (int)((int64_t)c * items / ctas); }
+// Split of the items over the CTAs.  A change of unit inside a CTA's range costs about as much as a few tiles (the
+// accumulators drain, the new unit's normalisers are merged from the partials, Q is reloaded), so what the CTAs
+// get equal shares of is  items + pen * (changes of unit): item i of the o-th non-empty unit sits at
+// v = i + pen * o, and CTA c takes the items with v in [c V / ctas, (c + 1) V / ctas).  `pen` stays below the
+// share of a CTA, so no CTA's range is empty.
+constexpr int kUnitChangeTiles = 3;
+struct Split {
+    int items, ctas, pen, Hkv;
+    int64_t V;
+};
+
+__device__ inline Split make_split(const SeqView &sv, int B, int Hkv, int grid)
+{
+    Split sp;
+    sp.Hkv = Hkv;
+    sp.items = sv.tiles[B] * Hkv;
+    sp.ctas = max(1, min(grid, sp.items));
+    sp.pen = max(0, min(kUnitChangeTiles, sp.items / sp.ctas - 1));
+    sp.V = (int64_t)sp.items + (int64_t)sp.pen * max(0, sv.ne[B] * Hkv - 1);
+    return sp;
+}
+
+// first item of CTA c (c == ctas: one past the last item)
+__device__ inline int range_begin(const Split &sp, const SeqView &sv, int B, int c)
+{
+    const int64_t t = ((int64_t)c * sp.V + sp.ctas - 1) / sp.ctas;      // smallest v of the CTA's share
+    if (t >= sp.V) return sp.items;
+    const int Hkv = sp.Hkv;
+    auto key = [&](int q) { return (int64_t)sv.tiles[q] * Hkv + (int64_t)sp.pen * sv.ne[q] * Hkv; };   // v of a sequence's first item
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (key(mid) <= t) lo = mid; else hi = mid;
+    }
+    const int nt = sv.tiles[lo + 1] - sv.tiles[lo];
+    const int64_t rel = t - key(lo);
+    const int g = (int)min((int64_t)(Hkv - 1), rel / (nt + sp.pen));
+    const int64_t r = rel - (int64_t)g * (nt + sp.pen);
+    // a v that falls between two units belongs to the first item of the second
+    return sv.tiles[lo] * Hkv + g * nt + (int)min(r, (int64_t)nt);
+}
+
+// CTA that owns item x of unit u
+__device__ inline int cta_of_item(const Split &sp, const SeqView &sv, int x, int u)
+{
+    const int ord = sv.ne[u / sp.Hkv] * sp.Hkv + u % sp.Hkv;
+    const int64_t v = (int64_t)x + (int64_t)sp.pen * ord;
+    return (int)min((int64_t)(sp.ctas - 1), v * sp.ctas / sp.V);
+}
 
 struct TcArgs {
     refree_params p;
@@ -708,21 +756,15 @@ __device__ inline float col_job(int nch, uint32_t taddr, uint64_t *empty_bar, in
     return s0 + s1;
 }
 
-// CTA that owns item x when `items` are split evenly over `ctas` (ctas <= items).
-__device__ inline int cta_of_item(int x, int items, int ctas)
-{
-    return (int)((((int64_t)x + 1) * ctas - 1) / items);
-}
-
 // L[row] = log2 sum over the row of 2^y for the rows of unit u, merged from the (reference, sum) pairs that pass 1
 // left per (CTA, unit, column half), in ascending record order (the same in every CTA that needs the unit).
 // Called by all epilogue threads; `ib` = index of the unit's first item, `ts` = its tiles.
-__device__ inline bool merge_unit_lse(const TcArgs &a, TcSmemTail &tl, int u, int ib, int ts, int items, int ctas,
-                                      uint32_t &ephase)
+__device__ inline bool merge_unit_lse(const TcArgs &a, TcSmemTail &tl, const SeqView &sv, const Split &sp, int u, int ib,
+                                      int ts, uint32_t &ephase)
 {
     const TcShape &sh = a.sh;
     const int tid = threadIdx.x;
-    const int c_lo = cta_of_item(ib, items, ctas), c_hi = cta_of_item(ib + ts - 1, items, ctas);
+    const int c_lo = cta_of_item(sp, sv, ib, u), c_hi = cta_of_item(sp, sv, ib + ts - 1, u);
     if (a.flags) {
         // one launch for both passes: the partials of this unit come from CTAs that may still be in pass 1;
         // wait (bounded) until each of them has published
@@ -785,7 +827,7 @@ __device__ inline bool merge_unit_lse(const TcArgs &a, TcSmemTail &tl, int u, in
 // (lane quarter) x (half of the product's columns); it leaves its share of the tile's column sums in a staging
 // slot, and the finishing warp adds the shares.
 __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const SeqView &sv, uint32_t tmem_base,
-                                      int item0, int nitems, int items, int ctas, EpiState &es)
+                                      int item0, int nitems, const Split &sp, EpiState &es)
 {
     const TcShape &sh = a.sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -809,7 +851,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
             // for the tile either: the partials come from the row pass, not from anything this pass loads.
             const ItemTc it = decode_item_tc(sv, a.p.num_seqs, a.p.num_kv_heads, item0 + (nitems - 1 - item));
             if (item > 0 && !(ok = epi_sync(tl, ephase))) break;   // nobody still reads the previous unit's L
-            ok = merge_unit_lse(a, tl, it.u, sv.tiles[it.s] * a.p.num_kv_heads + it.g * it.ntiles, it.ntiles, items, ctas,
+            ok = merge_unit_lse(a, tl, sv, sp, it.u, sv.tiles[it.s] * a.p.num_kv_heads + it.g * it.ntiles, it.ntiles,
                                 ephase);
             if (!ok) break;
             next_change = item + it.tile + 1;                      // the unit's earlier tiles follow
@@ -1062,7 +1104,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
     int32_t *tab = reinterpret_cast<int32_t *>(&tl + 1);
     const int B = a.p.num_seqs;
     int32_t *t_pack = tab, *t_tiles = tab + (B + 1), *t_len = tab + 2 * (B + 1), *t_start = tab + 2 * (B + 1) + B;
-    int32_t *coff = tab + 4 * B + 2;             // row copy: running sum of the budgets, units + 1 entries
+    int32_t *t_ne = tab + 4 * B + 2;
+    int32_t *coff = tab + 5 * B + 3;             // row copy: running sum of the budgets, units + 1 entries
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == kEpiWarps * 32) {
@@ -1092,17 +1135,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
     }
     for (int t = threadIdx.x; t < B; t += kThreadsTc) t_start[t] = a.seq_start[t];
     if (threadIdx.x == 32) {
-        int32_t pa = 0, ti = 0;
+        int32_t pa = 0, ti = 0, ne = 0;
         for (int s = 0; s < B; ++s) {
             t_pack[s] = pa;
             t_tiles[s] = ti;
+            t_ne[s] = ne;
             const int n = max(a.seq_len[s], 0);
             t_len[s] = n;
             pa += n;
             ti += ceil_div(n, kTile);
+            ne += n > 0 ? 1 : 0;
         }
         t_pack[B] = pa;
         t_tiles[B] = ti;
+        t_ne[B] = ne;
     }
     if (warp == kEpiWarps + 1) tmem_alloc(&tl.tmem_base, 512);
     tc_fence_before();
@@ -1118,19 +1164,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         for (int t = threadIdx.x; t < B * a.p.num_kv_heads; t += kThreadsTc)
             if (a.seq_len[t / a.p.num_kv_heads] <= 0) a.sel_lengths[t] = 0;
     SeqView sv;
-    sv.pack = t_pack; sv.tiles = t_tiles; sv.len = t_len; sv.start = t_start;
+    sv.pack = t_pack; sv.tiles = t_tiles; sv.len = t_len; sv.start = t_start; sv.ne = t_ne;
 
     // ranges over min(grid, items) CTAs, so that every CTA that has a range has a non-empty one
-    const int items = t_tiles[B] * a.p.num_kv_heads;
-    const int ctas = max(1, min((int)gridDim.x, items));
-    const bool active = (int)blockIdx.x < ctas;
-    const int item0 = active ? range_begin(blockIdx.x, items, ctas) : 0;
-    const int item1 = active ? range_begin(blockIdx.x + 1, items, ctas) : 0;
+    const Split sp = make_split(sv, B, a.p.num_kv_heads, (int)gridDim.x);
+    const bool active = (int)blockIdx.x < sp.ctas && sp.items > 0;
+    const int item0 = active ? range_begin(sp, sv, B, blockIdx.x) : 0;
+    const int item1 = active ? range_begin(sp, sv, B, blockIdx.x + 1) : 0;
 
     const int nitems = item1 - item0;
     if (warp < kEpiWarps) {
         EpiState es;
-        if (MODE == 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, items, ctas, es);
+        if (MODE == 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, sp, es);
         if (P1) epilogue_pass1(a, tl, tmem_base, nitems, es);
         if (MODE == 3) {
             // publish: this CTA's partials are in memory
@@ -1139,7 +1184,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
             if (threadIdx.x == 0)
                 asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.flags + blockIdx.x), "r"(1u) : "memory");
         }
-        if (P2 && MODE != 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, items, ctas, es);
+        if (P2 && MODE != 4) epilogue_pass2(a, tl, sv, tmem_base, item0, nitems, sp, es);
     } else if (warp == kEpiWarps) {
         if (lane == 0) {
             RingState rs;
@@ -1211,7 +1256,7 @@ bool shape_for(const refree_params &p, TcShape &sh)
 size_t smem_bytes(const TcShape &sh, int num_seqs, int copy_slots = 0, int copy_units = 0)
 {
     return 1024 + (size_t)sh.Rpad * 256 + (size_t)sh.stages * kTileBytes + (size_t)copy_slots * kCopySlot +
-           sizeof(TcSmemTail) + (size_t)(4 * num_seqs + 2) * sizeof(int32_t) +
+           sizeof(TcSmemTail) + (size_t)(5 * num_seqs + 3) * sizeof(int32_t) +
            (copy_slots ? (size_t)(copy_units + 1) * sizeof(int32_t) : 0);
 }
 

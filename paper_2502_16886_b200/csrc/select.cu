@@ -26,6 +26,8 @@
 
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "refree_internal.cuh"
 #include "select_groups.cuh"
 
@@ -200,6 +202,11 @@ struct SelectSmem {
     float fbuf[kWarps + 1];
     unsigned int hcnt[256];
     u64 hsum[256];
+    unsigned int hcnt2[2][256];       // register-resident score ranking: the block's histogram of a level, read by
+    u64 hsum2[2][256];                // the cluster; two copies taken in turn, so that one exchange needs one barrier
+    u64 dsum[8];                      // ... and its digit search: totals of the eight warps that own the digits
+    unsigned int dcnt[8];
+    int dcand[8];
     unsigned int wcnt[kWarps][257];   // per-warp private histograms (padded: one bank per warp for a digit)
     u64 wsum[kWarps][257];
     int pack;
@@ -260,7 +267,7 @@ __device__ inline bool choose_fixed_point(UnitView &v, SelectSmem &sm, int32_t *
 
 __global__ void __launch_bounds__(kThreads)
 select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_len,
-                     int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status)
+                     int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status, int skip_upto)
 {
     extern __shared__ __align__(16) unsigned char select_smem_raw[];
     SelectSmem &sm = *reinterpret_cast<SelectSmem *>(select_smem_raw);
@@ -271,6 +278,7 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     const bool layer = p.scope == REFREE_SCOPE_LAYER;
     const int s = layer ? unit : unit / Hkv;
     const int g = layer ? 0 : unit % Hkv;
+    if (skip_upto > 0 && max(seq_len[s], 0) <= skip_upto) return;      // the register-resident kernel takes these (the whole cluster leaves)
     if (threadIdx.x == 0) {
         int a = 0;
         for (int t = 0; t < s; ++t) a += max(seq_len[t], 0);
@@ -436,6 +444,199 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
     }
 }
 
+// Score ranking per head (Section 4.4) for sequences short enough that a cluster holds every key in registers:
+// position (e * blocks + rank) * kThreads + thread is element e of a thread, E elements each.  Same rule, fixed
+// point and radix descent as select_budget_kernel; the scores are read once, and a level of the descent costs a
+// handful of block barriers and one cluster barrier.
+template <int E>
+__global__ void __launch_bounds__(kThreads)
+select_score_resident_kernel(refree_params p, const float *scores, const int32_t *seq_len,
+                             int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status)
+{
+    extern __shared__ __align__(16) unsigned char select_smem_raw[];
+    SelectSmem &sm = *reinterpret_cast<SelectSmem *>(select_smem_raw);
+    cg::cluster_group cl = cg::this_cluster();
+    const int nblk = (int)cl.num_blocks(), rank = (int)cl.block_rank();
+    const int unit = blockIdx.x / nblk;
+    const int Hkv = p.num_kv_heads;
+    const int s = unit / Hkv, g = unit % Hkv;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        int a = 0;
+        for (int t = 0; t < s; ++t) a += max(seq_len[t], 0);
+        sm.pack = a;
+    }
+    __syncthreads();
+    const int n = max(seq_len[s], 0);
+    if (n > nblk * kThreads * E) return;             // too long to hold: select_budget_kernel takes it
+    UnitView v;
+    v.sc = scores + (int64_t)g * total_tokens + sm.pack;
+    v.head_stride = total_tokens;
+    v.heads = 1;
+    v.n = n;
+    v.w_eff = min(p.window, n);
+    v.lead = min(p.sink, n);
+    v.sbias = 0;
+    const int floor_b = p.keep_window ? min(n, v.lead + v.w_eff) : min(n, 1);
+    Cut cut;
+    cut.b = n; cut.ties = 0; cut.tau = 0; cut.prot_kept = 0; cut.sbias = 0;
+
+    uint32_t kb[E];                              // |score| bits; 0 past the sequence
+    uint32_t mx = 0;
+    bool bad = false;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int i = (e * nblk + rank) * kThreads + threadIdx.x;
+        kb[e] = i < n ? mag_bits(v.sc[i]) : 0u;
+        if ((kb[e] >> 23) == 255u) bad = true; else mx = max(mx, kb[e]);
+    }
+    if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
+    mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
+    mx = cluster_combine<uint32_t>(cl, &sm.x_u32, mx, MaxOpU());
+    if (n > 0 && mx != 0u) {
+        // fixed point of the unit: C_n * 2^S in [2^60, 2^61), from the binary order of magnitude of the sum of squares
+        const int emax = max(1, (int)(mx >> 23));
+        const float f = ldexpf(1.0f, 127 - emax);
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const float a = ((kb[e] >> 23) == 255u) ? 0.f : __uint_as_float(kb[e]) * f;
+            acc = fmaf(a, a, acc);
+        }
+        acc = block_reduce<float>(acc, sm.fbuf, AddOpF());
+        acc = cluster_combine<float>(cl, &sm.x_f32, acc, AddOpF());
+        v.sbias = 60 - ilogbf(fmaxf(acc, 0.25f)) - 2 * (emax - 127) - 300;
+        cut.sbias = v.sbias;
+        if (v.lead + v.w_eff >= n) { v.lead = n; v.w_eff = 0; }      // the protected prefix covers the sequence
+        const int prot = v.lead + v.w_eff;
+        u64 Cn;
+        {
+            u64 local = 0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) local += sq_fixed(kb[e], v.sbias);
+            u64 tot;
+            block_excl_scan<u64>(local, sm.ubuf, tot);
+            Cn = cluster_combine<u64>(cl, &sm.x_u64, tot, AddOpU64());
+        }
+        if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
+        __syncthreads();
+        const u64 c_min = sm.c_min;
+        const u64 Sprot = range_totals(v, 0, prot, ProtRank(), sm.wpre);
+        const int jp = range_find(v, prot, ProtRank(), c_min, sm.wpre, sm.ibuf);
+        int jstar = n;
+        cut.prot_kept = prot;
+        cut.tau = 0ull;                       // keep every unprotected position ...
+        cut.ties = INT_MAX;                   // ... unless a crossing is found below
+        if (jp != INT_MAX) {
+            jstar = jp;
+        } else if (prot < n && c_min != ~0ull) {
+            const u64 need = c_min - Sprot;   // mass still missing after the protected prefix (> 0)
+            uint32_t prefix = 0u, above_cnt = 0u;     // the same in every thread of the cluster
+            u64 above_sum = 0ull;
+            int digit_cnt = 0;
+            bool any = true;
+            for (int level = 0; level < 4 && any; ++level) {
+                const int shift = 24 - 8 * level;
+                const int hb = level & 1;
+                for (int t = threadIdx.x; t < kWarps * 257; t += kThreads) {
+                    (&sm.wcnt[0][0])[t] = 0u;
+                    (&sm.wsum[0][0])[t] = 0ull;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const int i = (e * nblk + rank) * kThreads + threadIdx.x;
+                    if (i >= v.lead && i < n - v.w_eff && (level == 0 || (kb[e] >> (shift + 8)) == prefix)) {
+                        const int dgt = (int)((kb[e] >> shift) & 255u);
+                        atomicAdd(&sm.wcnt[warp][dgt], 1u);
+                        atomicAdd(&sm.wsum[warp][dgt], sq_fixed(kb[e], v.sbias));
+                    }
+                }
+                __syncthreads();
+                if (threadIdx.x < 256) {
+                    unsigned int c = 0u;
+                    u64 sumv = 0ull;
+                    for (int wv = 0; wv < kWarps; ++wv) { c += sm.wcnt[wv][threadIdx.x]; sumv += sm.wsum[wv][threadIdx.x]; }
+                    sm.hcnt2[hb][threadIdx.x] = c;
+                    sm.hsum2[hb][threadIdx.x] = sumv;
+                }
+                // thread t < 256 owns digit 255 - t: the cluster's totals of it (integers: any order)
+                unsigned int mycnt = 0u;
+                u64 mysum = 0ull;
+                if (nblk > 1) {
+                    cl.sync();
+                    if (threadIdx.x < 256) {
+                        unsigned int rc[kMaxCluster];
+                        u64 rs[kMaxCluster];
+#pragma unroll
+                        for (int b = 0; b < kMaxCluster; ++b) {          // all remote reads in flight together
+                            rc[b] = b < nblk ? cl.map_shared_rank(sm.hcnt2[hb], b)[255 - threadIdx.x] : 0u;
+                            rs[b] = b < nblk ? cl.map_shared_rank(sm.hsum2[hb], b)[255 - threadIdx.x] : 0ull;
+                        }
+#pragma unroll
+                        for (int b = 0; b < kMaxCluster; ++b) { mycnt += rc[b]; mysum += rs[b]; }
+                    }
+                } else {
+                    __syncthreads();
+                    if (threadIdx.x < 256) { mycnt = sm.hcnt2[hb][255 - threadIdx.x]; mysum = sm.hsum2[hb][255 - threadIdx.x]; }
+                }
+                // sums from the top digit down; the first digit at which they reach what is missing
+                const u64 inc_s = warp_incl_scan(mysum);
+                const unsigned int inc_c = warp_incl_scan(mycnt);
+                if (warp < 8 && lane == 31) { sm.dsum[warp] = inc_s; sm.dcnt[warp] = inc_c; }
+                __syncthreads();
+                u64 abv_s = inc_s - mysum;
+                unsigned int abv_c = inc_c - mycnt;
+                if (warp < 8)
+                    for (int wv = 0; wv < warp; ++wv) { abv_s += sm.dsum[wv]; abv_c += sm.dcnt[wv]; }
+                const bool hit = warp < 8 && mycnt > 0u && above_sum + abv_s + mysum >= need;
+                const unsigned int hm = __ballot_sync(0xffffffffu, hit);
+                if (warp < 8 && lane == 0) sm.dcand[warp] = hm ? warp * 32 + __ffs(hm) - 1 : INT_MAX;
+                __syncthreads();
+                int cand = INT_MAX;
+                for (int wv = 0; wv < 8; ++wv) cand = min(cand, sm.dcand[wv]);
+                if ((int)threadIdx.x == cand) {
+                    sm.prefix = (u64)((prefix << 8) | (uint32_t)(255 - cand));
+                    sm.above_sum = above_sum + abv_s;
+                    sm.above_cnt = above_cnt + abv_c;
+                    sm.digit = (int)mycnt;
+                }
+                __syncthreads();
+                if (cand == INT_MAX) {
+                    any = false;              // the rule is never met: keep all
+                } else {
+                    prefix = (uint32_t)sm.prefix;
+                    above_sum = sm.above_sum;
+                    above_cnt = sm.above_cnt;
+                    digit_cnt = sm.digit;
+                }
+            }
+            if (any) {
+                // `prefix` is the key at which the sum crosses; digit_cnt positions share it
+                const u64 tau = (u64)prefix << 32;
+                const u64 fq = sq_fixed(prefix, v.sbias);
+                const u64 miss = need - above_sum;            // > 0: the digits above did not reach it
+                u64 t = fq ? (miss + fq - 1) / fq : 1ull;
+                t = max(1ull, min(t, (u64)digit_cnt));
+                jstar = prot + (int)above_cnt + (int)t;
+                cut.tau = tau;
+                cut.ties = (int)t;
+            }
+        }
+        cut.b = max(jstar, floor_b);
+        if (cut.b <= prot) {                 // nothing beyond the protected prefix
+            cut.prot_kept = cut.b;
+            cut.tau = ~0ull;
+            cut.ties = 0;
+        }
+    }
+    if (nblk > 1) cl.sync();               // no block exits while another may still read its shared memory
+    if (threadIdx.x == 0 && rank == 0) {
+        lengths[s * Hkv + g] = cut.b;
+        cuts[s * Hkv + g] = cut;
+    }
+}
+
 // Position ranking, one budget per (sequence, KV head), from the per-32-position
 // partials that the scoring kernel left (GroupPartial): the stopping rule then
 // touches one record per 32 scores plus the 32 scores of the group in which the
@@ -595,7 +796,9 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
             dst[t] = t < head ? t : n - b + t;
         return;
     }
-    if (blockIdx.x != 0) return;
+    // Score ranking: block c of the unit owns positions [c * kThreads, (c + 1) * kThreads), one per thread.
+    const int chunk = blockIdx.x * kThreads;
+    if (chunk >= n) return;
     if (threadIdx.x == 0) {
         int a = 0;
         for (int t = 0; t < s; ++t) a += max(seq_len[t], 0);
@@ -610,59 +813,55 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     v.heads = layer ? Hkv : 1;
     v.n = n; v.lead = lead; v.w_eff = w_eff;
     v.sbias = cut.sbias;
-    // Every warp owns a range of consecutive positions and walks it 32 at a time (coalesced loads);
-    // votes give the order inside a step, running counts the order inside the warp, and two block
-    // scans over the warps' totals the order inside the unit: ties first (which of the positions at
-    // the crossing key are kept: the lowest indices), then the kept positions.
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int span = ceil_div(ceil_div(n, kWarps), 32) * 32;
-    const int lo = min(n, warp * span), hi = min(n, lo + span);
-    auto classify = [&](int i, bool &sure, bool &tie) {
+    // kept for sure (above the crossing key, or protected and inside the budget) / at the crossing key, of
+    // which the cut.ties lowest positions are kept
+    // the key is loaded first, without a branch around it, so that a thread's loads are in flight together
+    auto key_of = [&](int i) { return (i >= lead && i < n - w_eff) ? key_at(v, i) : 0ull; };
+    auto classify = [&](int i, u64 key, bool &sure, bool &tie) {
         sure = false; tie = false;
-        if (i >= hi) return;
+        if (i >= n) return;
         if (i < lead) {
             sure = i < cut.prot_kept;
         } else if (i >= n - w_eff) {
             sure = lead + (i - (n - w_eff)) < cut.prot_kept;
         } else {
-            const u64 key = key_at(v, i);
             sure = key > cut.tau;
             tie = key == cut.tau;
         }
     };
-    int ties = 0;
-    for (int i0 = lo; i0 < hi; i0 += 32) {
-        bool sure, tie;
-        classify(i0 + lane, sure, tie);
-        ties += __popc(__ballot_sync(0xffffffffu, tie));
+    // what the positions before the chunk contribute: every block counts them itself (the scores are in L2)
+    long long before = 0;                                   // (sure << 32) + ties
+    for (int i0 = threadIdx.x; i0 < chunk; i0 += 8 * kThreads) {
+        u64 key[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) key[q] = key_of(i0 + q * kThreads < chunk ? i0 + q * kThreads : n);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            bool sure, tie;
+            classify(i0 + q * kThreads < chunk ? i0 + q * kThreads : n, key[q], sure, tie);
+            before += ((long long)sure << 32) + (long long)tie;
+        }
     }
-    int tie_tot, keep_tot;
-    const int tie_base = block_excl_scan<int>(lane == 0 ? ties : 0, ibuf, tie_tot);   // lane 0 carries the warp's count
-    int tie_rank = __shfl_sync(0xffffffffu, tie_base, 0);
-    const int tie_rank0 = tie_rank;
-    int keeps = 0;
-    for (int i0 = lo; i0 < hi; i0 += 32) {
-        bool sure, tie;
-        classify(i0 + lane, sure, tie);
-        const unsigned int tm = __ballot_sync(0xffffffffu, tie);
-        if (tie && tie_rank + __popc(tm & ((1u << lane) - 1u)) < cut.ties) sure = true;
-        tie_rank += __popc(tm);
-        keeps += __popc(__ballot_sync(0xffffffffu, sure));
+    {
+        long long tot;
+        block_excl_scan<long long>(before, lbuf, tot);
+        before = tot;
     }
-    const int keep_base = block_excl_scan<int>(lane == 0 ? keeps : 0, ibuf, keep_tot);
-    int slot = __shfl_sync(0xffffffffu, keep_base, 0);
-    tie_rank = tie_rank0;
-    for (int i0 = lo; i0 < hi; i0 += 32) {
-        bool sure, tie;
-        classify(i0 + lane, sure, tie);
-        const unsigned int tm = __ballot_sync(0xffffffffu, tie);
-        if (tie && tie_rank + __popc(tm & ((1u << lane) - 1u)) < cut.ties) sure = true;
-        tie_rank += __popc(tm);
-        const unsigned int km = __ballot_sync(0xffffffffu, sure);
-        const int mine = slot + __popc(km & ((1u << lane) - 1u));
-        if (sure && mine < b) dst[mine] = i0 + lane;
-        slot += __popc(km);
-    }
+    const int ties_before = (int)(before & 0xffffffffll), sure_before = (int)(before >> 32);
+    const int lane = threadIdx.x & 31;
+    bool sure, tie;
+    classify(chunk + threadIdx.x, key_of(chunk + threadIdx.x), sure, tie);
+    const unsigned int tm = __ballot_sync(0xffffffffu, tie);
+    int tie_tot;
+    const int tie_base = block_excl_scan<int>(lane == 0 ? __popc(tm) : 0, ibuf, tie_tot);   // lane 0 carries the warp's count
+    const int tie_rank = ties_before + __shfl_sync(0xffffffffu, tie_base, 0) + __popc(tm & ((1u << lane) - 1u));
+    if (tie && tie_rank < cut.ties) sure = true;
+    const unsigned int km = __ballot_sync(0xffffffffu, sure);
+    int keep_tot;
+    const int keep_base = block_excl_scan<int>(lane == 0 ? __popc(km) : 0, ibuf, keep_tot);
+    const int mine = sure_before + min(ties_before, cut.ties) + __shfl_sync(0xffffffffu, keep_base, 0) +
+                     __popc(km & ((1u << lane) - 1u));
+    if (sure && mine < b) dst[mine] = chunk + threadIdx.x;
 }
 
 }  // namespace
@@ -675,17 +874,30 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
     Cut *cuts = reinterpret_cast<Cut *>(ws + lay.cut_off);
     const int U = p.num_seqs * p.num_kv_heads;
     const int sel_units = p.scope == REFREE_SCOPE_LAYER ? p.num_seqs : U;
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
-        const cudaError_t e = cudaFuncSetAttribute(select_budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)sizeof(SelectSmem));
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
+    {
+        // the kernels' shared memory is above the default limit: raised once per device, under a lock
+        static std::mutex attr_mutex;
+        static bool attr_set[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> hold(attr_mutex);
+        if (!attr_set[dev]) {
+            const int bytes = (int)sizeof(SelectSmem);
+            cudaError_t e = cudaFuncSetAttribute(select_budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(select_score_resident_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(select_score_resident_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(select_score_resident_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e != cudaSuccess) return e;
+            attr_set[dev] = true;
+        }
     }
-    if (groups && p.rank_mode == REFREE_RANK_POSITION && p.scope == REFREE_SCOPE_HEAD && !p.force_full)
+    if (groups && p.rank_mode == REFREE_RANK_POSITION && p.scope == REFREE_SCOPE_HEAD && !p.force_full) {
         select_groups_kernel<<<U, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, groups, lengths, cuts);
-    else {
+        count_launches(1);
+    } else {
         // score ranking walks every score several times: a cluster of blocks shares a unit (distributed
         // shared memory for the few totals they exchange); position ranking keeps one block per unit
         int nblk = 1;
@@ -714,23 +926,59 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
                 attr[0].val.clusterDim.x = 1;
             }
         }
-        const cudaError_t le = cudaLaunchKernelEx(&cfg, select_budget_kernel, p, scores, seq_len, total_tokens, lengths,
-                                                  cuts, dev_status);
-        if (le != cudaSuccess) return le;
+        // Score ranking per head: units short enough for a cluster to hold in registers go to the kernel that
+        // reads the scores once; the general kernel takes the rest (all of them when none is short enough).
+        int skip_upto = 0;
+        if (p.rank_mode == REFREE_RANK_SCORE && !p.force_full && p.scope == REFREE_SCOPE_HEAD) {
+            int rb = nblk;                                   // blocks per unit: at least what the sizes call for
+            const int64_t want = std::min<int64_t>(total_tokens, (int64_t)kMaxCluster * kThreads * 16);
+            while (rb < kMaxCluster && (int64_t)rb * kThreads * 16 < want) rb *= 2;
+            int E = 4;
+            while (E < 16 && (int64_t)rb * kThreads * E < want) E *= 2;
+            cudaLaunchConfig_t rc = cfg;
+            cudaLaunchAttribute rattr[1];
+            rattr[0] = attr[0];
+            rattr[0].val.clusterDim.x = rb;
+            rc.attrs = rattr;
+            rc.gridDim = dim3(sel_units * rb);
+            cudaError_t re = cudaErrorInvalidValue;
+            int clusters = 0;
+            auto fits = [&](auto kern) {
+                return rb == 1 || (cudaOccupancyMaxActiveClusters(&clusters, kern, &rc) == cudaSuccess && clusters >= 1);
+            };
+            if (E == 4 && fits(select_score_resident_kernel<4>))
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<4>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+            else if (E == 8 && fits(select_score_resident_kernel<8>))
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<8>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+            else if (E == 16 && fits(select_score_resident_kernel<16>))
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<16>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+            if (re == cudaSuccess) {
+                skip_upto = rb * kThreads * E;
+                count_launches(1);
+            } else {
+                (void)cudaGetLastError();
+            }
+        }
+        if (skip_upto == 0 || (int64_t)skip_upto < total_tokens) {
+            const cudaError_t le = cudaLaunchKernelEx(&cfg, select_budget_kernel, p, scores, seq_len, total_tokens, lengths,
+                                                      cuts, dev_status, skip_upto);
+            if (le != cudaSuccess) return le;
+            count_launches(1);
+        }
     }
-    if (!emit) {               // the caller forms the offsets itself and needs no index list
-        count_launches(1);
-        return cudaGetLastError();
-    }
+    if (!emit) return cudaGetLastError();               // the caller forms the offsets itself and needs no index list
     const bool ranges = p.rank_mode == REFREE_RANK_POSITION || p.force_full;
     int gx = 1;
     if (ranges && kept_idx) {
         const int64_t per_unit = std::max<int64_t>(1, total_tokens / std::max(1, p.num_seqs));
         gx = (int)std::min<int64_t>(16, (per_unit + 4 * kThreads - 1) / (4 * kThreads));
+    } else if (kept_idx) {
+        // score ranking: a block per kThreads positions of the longest sequence there can be
+        gx = (int)std::max<int64_t>(1, (total_tokens + kThreads - 1) / kThreads);
     }
     emit_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, offsets,
                                                   kept_idx, capacity_rows, dev_status);
-    count_launches(2);
+    count_launches(1);
     return cudaGetLastError();
 }
 

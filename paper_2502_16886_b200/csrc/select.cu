@@ -451,7 +451,8 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
 template <int E>
 __global__ void __launch_bounds__(kThreads)
 select_score_resident_kernel(refree_params p, const float *scores, const int32_t *seq_len,
-                             int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status)
+                             int64_t total_tokens, int32_t *lengths, Cut *cuts, int32_t *dev_status,
+                             int2 *chunk_counts, int chunk_stride)
 {
     extern __shared__ __align__(16) unsigned char select_smem_raw[];
     SelectSmem &sm = *reinterpret_cast<SelectSmem *>(select_smem_raw);
@@ -630,6 +631,34 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
             cut.ties = 0;
         }
     }
+    if (chunk_counts) {
+        // For the kernel that writes the index list: per run of kThreads positions, how many are kept for sure
+        // and how many sit at the crossing key (element e of this block is run e * blocks + rank).
+        const int lead = v.lead, w_eff = v.w_eff;
+        int *wc = reinterpret_cast<int *>(&sm.wcnt[0][0]);              // [E][kWarps][2], free after the descent
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int i = (e * nblk + rank) * kThreads + threadIdx.x;
+            bool sure = false, tie = false;
+            if (i < n) {
+                if (i < lead) sure = i < cut.prot_kept;
+                else if (i >= n - w_eff) sure = lead + (i - (n - w_eff)) < cut.prot_kept;
+                else { const u64 key = (u64)kb[e] << 32; sure = key > cut.tau; tie = key == cut.tau; }
+            }
+            const unsigned int smask = __ballot_sync(0xffffffffu, sure), tmask = __ballot_sync(0xffffffffu, tie);
+            if (lane == 0) { wc[(e * kWarps + warp) * 2] = __popc(smask); wc[(e * kWarps + warp) * 2 + 1] = __popc(tmask); }
+        }
+        __syncthreads();
+        if (threadIdx.x < E) {
+            const int e = threadIdx.x, c = e * nblk + rank;
+            if ((int64_t)c * kThreads < n) {
+                int sure = 0, ties = 0;
+                for (int wv = 0; wv < kWarps; ++wv) { sure += wc[(e * kWarps + wv) * 2]; ties += wc[(e * kWarps + wv) * 2 + 1]; }
+                chunk_counts[(int64_t)(s * Hkv + g) * chunk_stride + c] = make_int2(sure, ties);
+            }
+        }
+    }
     if (nblk > 1) cl.sync();               // no block exits while another may still read its shared memory
     if (threadIdx.x == 0 && rank == 0) {
         lengths[s * Hkv + g] = cut.b;
@@ -761,7 +790,7 @@ select_groups_kernel(refree_params p, const float *scores, const int32_t *seq_le
 __global__ void __launch_bounds__(kThreads)
 emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_t total_tokens,
             const int32_t *lengths, const Cut *cuts, int64_t *offsets, int32_t *kept_idx,
-            int64_t capacity_rows, int32_t *dev_status)
+            int64_t capacity_rows, int32_t *dev_status, const int2 *chunk_counts, int chunk_stride, int counted_upto)
 {
     __shared__ long long lbuf[kWarps + 1];
     __shared__ int ibuf[kWarps + 1];
@@ -816,7 +845,15 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     // kept for sure (above the crossing key, or protected and inside the budget) / at the crossing key, of
     // which the cut.ties lowest positions are kept
     // the key is loaded first, without a branch around it, so that a thread's loads are in flight together
-    auto key_of = [&](int i) { return (i >= lead && i < n - w_eff) ? key_at(v, i) : 0ull; };
+    const bool one_head = v.heads == 1;
+    auto key_of = [&](int i) {
+        if (one_head) {                           // a plain predicated load, so the loads of an unrolled loop overlap
+            const int ic = min(max(i, 0), n - 1);
+            const uint32_t bits = mag_bits(v.sc[ic]);
+            return (i >= lead && i < n - w_eff) ? (u64)bits << 32 : 0ull;
+        }
+        return (i >= lead && i < n - w_eff) ? key_at(v, i) : 0ull;
+    };
     auto classify = [&](int i, u64 key, bool &sure, bool &tie) {
         sure = false; tie = false;
         if (i >= n) return;
@@ -829,8 +866,15 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
             tie = key == cut.tau;
         }
     };
-    // what the positions before the chunk contribute: every block counts them itself (the scores are in L2)
+    // What the positions before the chunk contribute: left per run of kThreads positions by the kernel that chose
+    // the budget when it held the unit in registers; otherwise every block counts them itself (the scores are in L2).
     long long before = 0;                                   // (sure << 32) + ties
+    if (chunk_counts && n <= counted_upto) {
+        for (int c = threadIdx.x; c < (int)blockIdx.x; c += kThreads) {
+            const int2 cc = chunk_counts[(int64_t)u * chunk_stride + c];
+            before += ((long long)cc.x << 32) + (long long)cc.y;
+        }
+    } else
     for (int i0 = threadIdx.x; i0 < chunk; i0 += 8 * kThreads) {
         u64 key[8];
 #pragma unroll
@@ -894,6 +938,9 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
             attr_set[dev] = true;
         }
     }
+    int skip_upto = 0;                       // units up to this length went to the register-resident kernel
+    int2 *chunk_counts = nullptr;
+    const int chunk_stride = (int)((total_tokens + kThreads - 1) / kThreads) + 1;
     if (groups && p.rank_mode == REFREE_RANK_POSITION && p.scope == REFREE_SCOPE_HEAD && !p.force_full) {
         select_groups_kernel<<<U, kThreads, 0, st>>>(p, scores, seq_len, total_tokens, groups, lengths, cuts);
         count_launches(1);
@@ -928,7 +975,6 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
         }
         // Score ranking per head: units short enough for a cluster to hold in registers go to the kernel that
         // reads the scores once; the general kernel takes the rest (all of them when none is short enough).
-        int skip_upto = 0;
         if (p.rank_mode == REFREE_RANK_SCORE && !p.force_full && p.scope == REFREE_SCOPE_HEAD) {
             int rb = nblk;                                   // blocks per unit: at least what the sizes call for
             const int64_t want = std::min<int64_t>(total_tokens, (int64_t)kMaxCluster * kThreads * 16);
@@ -946,17 +992,21 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
             auto fits = [&](auto kern) {
                 return rb == 1 || (cudaOccupancyMaxActiveClusters(&clusters, kern, &rc) == cudaSuccess && clusters >= 1);
             };
+            // counts per run of kThreads positions for the index list, where the caller's workspace has room for them
+            if (emit && kept_idx && lay.part_bytes >= (size_t)U * (size_t)chunk_stride * sizeof(int2))
+                chunk_counts = reinterpret_cast<int2 *>(ws + lay.part_off);
             if (E == 4 && fits(select_score_resident_kernel<4>))
-                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<4>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<4>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status, chunk_counts, chunk_stride);
             else if (E == 8 && fits(select_score_resident_kernel<8>))
-                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<8>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<8>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status, chunk_counts, chunk_stride);
             else if (E == 16 && fits(select_score_resident_kernel<16>))
-                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<16>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status);
+                re = cudaLaunchKernelEx(&rc, select_score_resident_kernel<16>, p, scores, seq_len, total_tokens, lengths, cuts, dev_status, chunk_counts, chunk_stride);
             if (re == cudaSuccess) {
                 skip_upto = rb * kThreads * E;
                 count_launches(1);
             } else {
                 (void)cudaGetLastError();
+                chunk_counts = nullptr;
             }
         }
         if (skip_upto == 0 || (int64_t)skip_upto < total_tokens) {
@@ -977,7 +1027,7 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
         gx = (int)std::max<int64_t>(1, (total_tokens + kThreads - 1) / kThreads);
     }
     emit_kernel<<<dim3(gx, U), kThreads, 0, st>>>(p, scores, seq_len, total_tokens, lengths, cuts, offsets,
-                                                  kept_idx, capacity_rows, dev_status);
+                                                  kept_idx, capacity_rows, dev_status, chunk_counts, chunk_stride, skip_upto);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -206,7 +206,11 @@ struct SelectSmem {
     u64 hsum2[2][256];                // the cluster; two copies taken in turn, so that one exchange needs one barrier
     u64 dsum[8];                      // ... and its digit search: totals of the eight warps that own the digits
     unsigned int dcnt[8];
-    int dcand[8];
+    int dcand[8];                     // first digit of each of those warps at which the sum crosses, with what is
+    u64 dabv_s[8];                    // above it and how many share it
+    unsigned int dabv_c[8], ddig[8];
+    uint32_t y_mx;                    // fixed point, exchanged once: a block's largest key and its sum of squares
+    float y_acc;                      // at that key's scale
     unsigned int wcnt[kWarps][257];   // per-warp private histograms (padded: one bank per warp for a digit)
     u64 wsum[kWarps][257];
     int pack;
@@ -492,20 +496,42 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
         if ((kb[e] >> 23) == 255u) bad = true; else mx = max(mx, kb[e]);
     }
     if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
-    mx = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
-    mx = cluster_combine<uint32_t>(cl, &sm.x_u32, mx, MaxOpU());
-    if (n > 0 && mx != 0u) {
-        // fixed point of the unit: C_n * 2^S in [2^60, 2^61), from the binary order of magnitude of the sum of squares
-        const int emax = max(1, (int)(mx >> 23));
-        const float f = ldexpf(1.0f, 127 - emax);
-        float acc = 0.f;
+    // Fixed point of the unit: C_n * 2^S in [2^60, 2^61), from the binary order of magnitude of the sum of squares.
+    // A block sums its squares at the scale of its own largest key; the blocks exchange (largest key, sum) once and
+    // bring the sums to the scale of the unit's largest key, a power of two apart, in rank order.
+    const uint32_t mx_b = block_reduce<uint32_t>(mx, reinterpret_cast<uint32_t *>(sm.ibuf), MaxOpU());
+    float acc_b = 0.f;
+    {
+        const float fb = ldexpf(1.0f, 127 - max(1, (int)(mx_b >> 23)));
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            const float a = ((kb[e] >> 23) == 255u) ? 0.f : __uint_as_float(kb[e]) * f;
-            acc = fmaf(a, a, acc);
+            const float a = ((kb[e] >> 23) == 255u) ? 0.f : __uint_as_float(kb[e]) * fb;
+            acc_b = fmaf(a, a, acc_b);
         }
-        acc = block_reduce<float>(acc, sm.fbuf, AddOpF());
-        acc = cluster_combine<float>(cl, &sm.x_f32, acc, AddOpF());
+        acc_b = block_reduce<float>(acc_b, sm.fbuf, AddOpF());
+    }
+    float acc = acc_b;
+    mx = mx_b;
+    if (nblk > 1) {
+        if (threadIdx.x == 0) { sm.y_mx = mx_b; sm.y_acc = acc_b; }
+        cl.sync();                                  // the slots are written once: no second barrier
+        uint32_t rm[kMaxCluster];
+        float ra[kMaxCluster];
+#pragma unroll
+        for (int b = 0; b < kMaxCluster; ++b) {
+            rm[b] = b < nblk ? *cl.map_shared_rank(&sm.y_mx, b) : 0u;
+            ra[b] = b < nblk ? *cl.map_shared_rank(&sm.y_acc, b) : 0.f;
+        }
+        mx = 0u;
+#pragma unroll
+        for (int b = 0; b < kMaxCluster; ++b) mx = max(mx, rm[b]);
+        acc = 0.f;
+#pragma unroll
+        for (int b = 0; b < kMaxCluster; ++b)
+            if (b < nblk) acc += ldexpf(ra[b], 2 * (max(1, (int)(rm[b] >> 23)) - max(1, (int)(mx >> 23))));
+    }
+    if (n > 0 && mx != 0u) {
+        const int emax = max(1, (int)(mx >> 23));
         v.sbias = 60 - ilogbf(fmaxf(acc, 0.25f)) - 2 * (emax - 127) - 300;
         cut.sbias = v.sbias;
         if (v.lead + v.w_eff >= n) { v.lead = n; v.w_eff = 0; }      // the protected prefix covers the sequence
@@ -517,11 +543,19 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
             for (int e = 0; e < E; ++e) local += sq_fixed(kb[e], v.sbias);
             u64 tot;
             block_excl_scan<u64>(local, sm.ubuf, tot);
-            Cn = cluster_combine<u64>(cl, &sm.x_u64, tot, AddOpU64());
+            Cn = tot;
+            if (nblk > 1) {
+                if (threadIdx.x == 0) sm.x_u64 = tot;
+                cl.sync();                              // written once: no second barrier
+                u64 rt[kMaxCluster];
+#pragma unroll
+                for (int b = 0; b < kMaxCluster; ++b) rt[b] = b < nblk ? *cl.map_shared_rank(&sm.x_u64, b) : 0ull;
+                Cn = 0ull;
+#pragma unroll
+                for (int b = 0; b < kMaxCluster; ++b) Cn += rt[b];
+            }
         }
-        if (threadIdx.x == 0) sm.c_min = crossing_level(Cn, (double)p.threshold);
-        __syncthreads();
-        const u64 c_min = sm.c_min;
+        const u64 c_min = crossing_level(Cn, (double)p.threshold);      // every thread: a handful of fp64 operations
         const u64 Sprot = range_totals(v, 0, prot, ProtRank(), sm.wpre);
         const int jp = range_find(v, prot, ProtRank(), c_min, sm.wpre, sm.ibuf);
         int jstar = n;
@@ -536,14 +570,17 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
             u64 above_sum = 0ull;
             int digit_cnt = 0;
             bool any = true;
-            for (int level = 0; level < 4 && any; ++level) {
-                const int shift = 24 - 8 * level;
-                const int hb = level & 1;
+            auto clear_hist = [&]() {
                 for (int t = threadIdx.x; t < kWarps * 257; t += kThreads) {
                     (&sm.wcnt[0][0])[t] = 0u;
                     (&sm.wsum[0][0])[t] = 0ull;
                 }
-                __syncthreads();
+            };
+            clear_hist();
+            __syncthreads();
+            for (int level = 0; level < 4 && any; ++level) {
+                const int shift = 24 - 8 * level;
+                const int hb = level & 1;
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
                     const int i = (e * nblk + rank) * kThreads + threadIdx.x;
@@ -581,6 +618,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
                     __syncthreads();
                     if (threadIdx.x < 256) { mycnt = sm.hcnt2[hb][255 - threadIdx.x]; mysum = sm.hsum2[hb][255 - threadIdx.x]; }
                 }
+                clear_hist();                 // for the next level: the per-warp histograms were read before the barrier above
                 // sums from the top digit down; the first digit at which they reach what is missing
                 const u64 inc_s = warp_incl_scan(mysum);
                 const unsigned int inc_c = warp_incl_scan(mycnt);
@@ -592,24 +630,27 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
                     for (int wv = 0; wv < warp; ++wv) { abv_s += sm.dsum[wv]; abv_c += sm.dcnt[wv]; }
                 const bool hit = warp < 8 && mycnt > 0u && above_sum + abv_s + mysum >= need;
                 const unsigned int hm = __ballot_sync(0xffffffffu, hit);
-                if (warp < 8 && lane == 0) sm.dcand[warp] = hm ? warp * 32 + __ffs(hm) - 1 : INT_MAX;
-                __syncthreads();
-                int cand = INT_MAX;
-                for (int wv = 0; wv < 8; ++wv) cand = min(cand, sm.dcand[wv]);
-                if ((int)threadIdx.x == cand) {
-                    sm.prefix = (u64)((prefix << 8) | (uint32_t)(255 - cand));
-                    sm.above_sum = above_sum + abv_s;
-                    sm.above_cnt = above_cnt + abv_c;
-                    sm.digit = (int)mycnt;
+                if (warp < 8) {
+                    const int first = hm ? __ffs(hm) - 1 : 0;
+                    if (lane == first) {          // the warp's first crossing digit leaves its record (none: lane 0 says so)
+                        sm.dcand[warp] = hm ? warp * 32 + first : INT_MAX;
+                        sm.dabv_s[warp] = abv_s;
+                        sm.dabv_c[warp] = abv_c;
+                        sm.ddig[warp] = mycnt;
+                    }
                 }
                 __syncthreads();
+                int cand = INT_MAX, cw = 0;
+#pragma unroll
+                for (int wv = 7; wv >= 0; --wv)
+                    if (sm.dcand[wv] != INT_MAX) { cand = sm.dcand[wv]; cw = wv; }
                 if (cand == INT_MAX) {
                     any = false;              // the rule is never met: keep all
                 } else {
-                    prefix = (uint32_t)sm.prefix;
-                    above_sum = sm.above_sum;
-                    above_cnt = sm.above_cnt;
-                    digit_cnt = sm.digit;
+                    prefix = (prefix << 8) | (uint32_t)(255 - cand);
+                    above_sum += sm.dabv_s[cw];
+                    above_cnt += sm.dabv_c[cw];
+                    digit_cnt = (int)sm.ddig[cw];
                 }
             }
             if (any) {

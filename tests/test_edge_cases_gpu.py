@@ -92,3 +92,48 @@ def test_score_ranking_with_eight_blocks_per_unit():
     lay = workloads.make_layer(cfg, 0, seq_lens=[40000])
     parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE)
     parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE, scope=binding.SCOPE_LAYER, threshold=0.05)
+
+
+def test_score_ranking_with_units_on_both_sides_of_what_a_cluster_holds_in_registers():
+    # score ranking per head keeps a unit's keys in the registers of a cluster of blocks when they fit
+    # (8 blocks x 1024 threads x 16 keys); here one sequence is longer than that and goes to the kernel
+    # that re-reads the scores, the others do not, and the index list is written for both kinds in one launch
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1, window=16, heavy_count=300)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[140_000, 700, 9000])
+    parity.run_fused_and_check(cfg, lay, rank_mode=binding.RANK_SCORE)
+
+
+@pytest.mark.parametrize("n", [1023, 1024, 1025, 4096, 20_000])
+def test_score_ranking_with_many_equal_scores_at_the_crossing(n):
+    # equal scores at the crossing key: the lowest positions among them are kept, whatever run of 1024
+    # positions (one block of the kernel that writes the index list) they fall into
+    cfg = cfg_like(num_q_heads=2, num_kv_heads=1, window=4)
+    p = binding.Params(num_seqs=1, num_q_heads=2, num_kv_heads=1, head_dim=64, window=4, sink=2, threshold=0.3,
+                       rank_mode=binding.RANK_SCORE, dtype=binding.DTYPE_F32, kv_tokens=n,
+                       k_strides=(0, 64, n * 64), v_strides=(0, 64, n * 64))
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(n)
+    vals = torch.tensor([0.5, 0.25, 0.125, 0.0625])
+    scores = vals[torch.randint(0, 4, (1, n), generator=g)].contiguous()
+    sl = torch.tensor([n], dtype=torch.int32)
+    lengths = torch.zeros(1, dtype=torch.int32, device=dev)
+    offsets = torch.zeros(2, dtype=torch.int64, device=dev)
+    kept = torch.full((n,), -1, dtype=torch.int32, device=dev)
+    ws = torch.empty(binding.refree_workspace_size(p, n), dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.refree_select_budget(p, scores.to(dev), sl.to(dev), n, lengths, offsets, kept, n, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    b = int(lengths.item())
+    got = kept[:b].cpu().tolist()
+    # brute force: protected positions first, then by decreasing score, ties by position
+    a = scores[0].double().numpy()
+    prot = [0, 1] + list(range(n - 4, n))
+    rest = sorted((i for i in range(2, n - 4)), key=lambda i: (-a[i], i))
+    order = prot + rest
+    import numpy as np
+    c = np.cumsum(a[order] ** 2)
+    j = int(np.argmax(1.0 - np.sqrt(c / c[-1]) < 0.3)) + 1
+    want_b = max(j, len(prot))
+    assert b == want_b
+    assert got == sorted(order[:b])

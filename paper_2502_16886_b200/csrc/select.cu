@@ -195,6 +195,18 @@ __device__ inline int range_find(const UnitView &v, int count, PosOf pos_of, u64
     return found;
 }
 
+// x += v for a 64-bit counter in shared memory, as two 32-bit atomic adds with the carry passed on (the halves
+// are only read together after a barrier).  Shared memory has 32-bit atomic adds in hardware; a 64-bit one is a
+// compare-and-swap loop, which crawls when most of a warp meets at one counter.
+__device__ inline void add_u64_shared(u64 *x, u64 v)
+{
+    uint32_t *h = reinterpret_cast<uint32_t *>(x);
+    const uint32_t lo = (uint32_t)v;
+    const uint32_t old = atomicAdd(h, lo);
+    const uint32_t hi = (uint32_t)(v >> 32) + (old + lo < old ? 1u : 0u);
+    if (hi) atomicAdd(h + 1, hi);
+}
+
 struct SelectSmem {
     u64 wpre[kWarps + 1];
     u64 ubuf[kWarps + 1];
@@ -371,7 +383,7 @@ select_budget_kernel(refree_params p, const float *scores, const int32_t *seq_le
                             if (i0 + q * kThreads < n - v.w_eff && (level == 0 || (key[q] >> (shift + 8)) == prefix)) {
                                 const int dgt = (int)((key[q] >> shift) & 255ull);
                                 atomicAdd(&sm.wcnt[warp][dgt], 1u);
-                                atomicAdd(&sm.wsum[warp][dgt], val[q]);
+                                add_u64_shared(&sm.wsum[warp][dgt], val[q]);
                             }
                         }
                     }
@@ -587,7 +599,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
                     if (i >= v.lead && i < n - v.w_eff && (level == 0 || (kb[e] >> (shift + 8)) == prefix)) {
                         const int dgt = (int)((kb[e] >> shift) & 255u);
                         atomicAdd(&sm.wcnt[warp][dgt], 1u);
-                        atomicAdd(&sm.wsum[warp][dgt], sq_fixed(kb[e], v.sbias));
+                        add_u64_shared(&sm.wsum[warp][dgt], sq_fixed(kb[e], v.sbias));
                     }
                 }
                 __syncthreads();

@@ -3,6 +3,7 @@
 // loads and stores, several rows in flight per thread.  Rows are copied bit for
 // bit.  With position ranking the kept set is two contiguous ranges, so the
 // source row follows from (b, m, n) and no index list is read.
+#include <mutex>
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -351,11 +352,13 @@ cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, con
         count_launches(1);
         return cudaGetLastError();
     }
+    static std::mutex grid_mutex;                 // the per-device grid size is looked up once, under a lock
     static int grid_blocks[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::unique_lock<std::mutex> hold(grid_mutex);
     if (grid_blocks[dev] == 0) {
         // every block of the grid must be resident at once: the rounds end in a grid-wide barrier
         int sms = 0, per_sm = 0, coop = 0;
@@ -367,11 +370,13 @@ cudaError_t launch_compact_inplace(const refree_params &p, void *k, void *v, con
         if (per_sm < 1) return cudaErrorLaunchOutOfResources;
         grid_blocks[dev] = sms * std::min(per_sm, 4);
     }
+    const int grid = grid_blocks[dev];
+    hold.unlock();
     refree_params pv = p;
     char *kc = (char *)k, *vc = (char *)v;
     int ranges = position_ranges ? 1 : 0;
     void *args[9] = {&pv, &kc, &vc, &seq_start, &seq_len, &offsets, &kept_idx, &ranges, &dev_status};
-    e = cudaLaunchCooperativeKernel((const void *)compact_inplace_kernel, dim3(grid_blocks[dev]), dim3(kThreads), args, 0, st);
+    e = cudaLaunchCooperativeKernel((const void *)compact_inplace_kernel, dim3(grid), dim3(kThreads), args, 0, st);
     if (e != cudaSuccess) return e;
     count_launches(1);
     return cudaGetLastError();

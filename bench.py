@@ -182,7 +182,7 @@ def algorithmic_bytes(cfg, seq_lens, lengths):
 # still has the hash it was captured on, and null afterwards.
 NCU_TRAFFIC = {
     # workload: (kernel source, first 16 hex digits of its sha256, bytes per launch)
-    "mistral7b_32k": ("paper_2502_16886_b200/csrc/score_tc.cu", "3b3723809f570add", 263_049_984 + 94_838_784),
+    "mistral7b_32k": ("paper_2502_16886_b200/csrc/score_tc.cu", "320db937c7063529", 262_295_296 + 97_656_320),
 }
 
 

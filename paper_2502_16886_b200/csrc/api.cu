@@ -334,7 +334,7 @@ static refree_status enqueue_layer(const refree_params *p, const void *q_win, co
     // sums of squares, and the stopping rule reads those instead of every score
     GroupPartial *groups = nullptr;
     if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
-        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
+        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0 && total_tokens <= kGroupSelectMaxTokens)
         groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
     if (total_tokens > 0 && (!p->force_full || scores))
         e = run_score(*p, q_win, k, seq_start, seq_len, total_tokens, sc, ws, lay, device_status, cs, groups);
@@ -404,7 +404,7 @@ refree_status refree_compress_layer_inplace(const refree_params *p, const void *
     int32_t *kept = ranges ? nullptr : reinterpret_cast<int32_t *>(ws + lay.kept_off);
     GroupPartial *groups = nullptr;
     if ((use_tc(*p, q_win) || score_w1_supported(*p)) && p->rank_mode == REFREE_RANK_POSITION &&
-        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0)
+        p->scope == REFREE_SCOPE_HEAD && !p->force_full && total_tokens > 0 && total_tokens <= kGroupSelectMaxTokens)
         groups = reinterpret_cast<GroupPartial *>(ws + lay.grp_off);
     cudaError_t e = cudaSuccess;
     if (total_tokens > 0 && !p->force_full)
@@ -501,7 +501,8 @@ refree_status refree_compress_layers(const refree_params *p, int32_t num_layers,
             t.k = k[l];
             t.ws = ws;
             t.scores = reinterpret_cast<float *>(ws + lay.scores_off);
-            t.groups = p->scope == REFREE_SCOPE_HEAD ? reinterpret_cast<GroupPartial *>(ws + lay.grp_off) : nullptr;
+            t.groups = p->scope == REFREE_SCOPE_HEAD && total_tokens <= kGroupSelectMaxTokens
+                           ? reinterpret_cast<GroupPartial *>(ws + lay.grp_off) : nullptr;
             t.sel_lengths = t.groups ? lengths[l] : nullptr;      // the rule runs inside the launch that finishes the layer
             return t;
         };

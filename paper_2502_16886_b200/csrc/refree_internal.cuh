@@ -15,6 +15,12 @@ constexpr int kMaxRows = 1024;   // G * window handled by the generic scoring pa
 
 // Bounded spin: polls before a wait gives up and reports REFREE_DEV_TIMEOUT.
 constexpr uint32_t kSpinLimit = 1u << 22;
+// The stopping rule fed by per-32-position records sums each group at a scale set by the group's own largest
+// score and shifts the sums to the unit's scale, so it drops up to one unit of the fixed point per element and per
+// group: about n * 2^(L - 54) of C_n with L = log2(groups), against n * 2^-60 for the rule that reads every score.
+// That is 2^-29 at 32K positions and still 2^-25 at 128K, far inside the near-tie band; longer sequences take the
+// rule that reads every score.
+constexpr int64_t kGroupSelectMaxTokens = 131072;
 
 // Layout of the caller-provided workspace.  All offsets are multiples of 256.
 struct Workspace {

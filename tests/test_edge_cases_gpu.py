@@ -137,3 +137,10 @@ def test_score_ranking_with_many_equal_scores_at_the_crossing(n):
     want_b = max(j, len(prot))
     assert b == want_b
     assert got == sorted(order[:b])
+
+
+def test_position_ranking_beyond_the_length_the_record_fed_rule_takes():
+    # above 131072 tokens in a call the budgets come from the rule that reads every score
+    cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1, window=16, heavy_count=300)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[140_000, 700])
+    parity.run_fused_and_check(cfg, lay)

@@ -113,3 +113,26 @@ def test_memory_probes_copy_the_rows_they_say(bulk):
     torch.cuda.synchronize()
     assert torch.equal(parity.bits(k_out), parity.bits(k[rows - kept:]))
     assert torch.equal(parity.bits(v_out), parity.bits(v[rows - kept:]))
+
+
+def test_record_fed_rule_equals_the_rule_that_reads_every_score_at_its_longest_sequence():
+    """131072 positions is the longest call whose budgets come from the per-32-position records; there its
+    coarser fixed point must still give the budgets of the rule that reads every score."""
+    cfg = dataclasses.replace(workloads.CONFIGS[1], num_layers=1, num_q_heads=4, num_kv_heads=2, window=16)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[131_072])
+    p = binding.params_for(cfg, lay)
+    total = lay.total_tokens
+    res = binding.compress_layer(p, lay.q_win.to(DEV), lay.k.to(DEV), lay.v.to(DEV), lay.seq_start.to(DEV),
+                                 lay.seq_len.to(DEV), total, want_scores=True, want_kept_idx=False)
+    torch.cuda.synchronize()
+    assert int(res.device_status.item()) == 0
+    units = p.num_seqs * p.num_kv_heads
+    lengths = torch.zeros(units, dtype=torch.int32, device=DEV)
+    offsets = torch.zeros(units + 1, dtype=torch.int64, device=DEV)
+    ws = torch.empty(binding.refree_workspace_size(p, total), dtype=torch.uint8, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.refree_select_budget(p, res.scores, lay.seq_len.to(DEV), total, lengths, offsets, None,
+                                 p.num_kv_heads * total, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    np.testing.assert_array_equal(lengths.cpu().numpy(), res.lengths.reshape(-1).cpu().numpy())

@@ -486,6 +486,9 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
     __syncthreads();
     const int n = max(seq_len[s], 0);
     if (n > nblk * kThreads * E) return;             // too long to hold: select_budget_kernel takes it
+    // elements of this block that lie inside the sequence: a batch sized for its longest sequence leaves most of
+    // a short one's element slots empty, and the loops below skip them (the same for every thread of the block)
+    const int e_lim = min(E, ceil_div(max(n - rank * kThreads, 0), nblk * kThreads));
     UnitView v;
     v.sc = scores + (int64_t)g * total_tokens + sm.pack;
     v.head_stride = total_tokens;
@@ -504,7 +507,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
 #pragma unroll
     for (int e = 0; e < E; ++e) {
         const int i = (e * nblk + rank) * kThreads + threadIdx.x;
-        kb[e] = i < n ? mag_bits(v.sc[i]) : 0u;
+        kb[e] = (e < e_lim && i < n) ? mag_bits(v.sc[i]) : 0u;
         if ((kb[e] >> 23) == 255u) bad = true; else mx = max(mx, kb[e]);
     }
     if (bad && dev_status) atomicOr(dev_status, REFREE_DEV_NONFINITE);
@@ -517,6 +520,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
         const float fb = ldexpf(1.0f, 127 - max(1, (int)(mx_b >> 23)));
 #pragma unroll
         for (int e = 0; e < E; ++e) {
+            if (e >= e_lim) continue;
             const float a = ((kb[e] >> 23) == 255u) ? 0.f : __uint_as_float(kb[e]) * fb;
             acc_b = fmaf(a, a, acc_b);
         }
@@ -552,7 +556,8 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
         {
             u64 local = 0;
 #pragma unroll
-            for (int e = 0; e < E; ++e) local += sq_fixed(kb[e], v.sbias);
+            for (int e = 0; e < E; ++e)
+                if (e < e_lim) local += sq_fixed(kb[e], v.sbias);
             u64 tot;
             block_excl_scan<u64>(local, sm.ubuf, tot);
             Cn = tot;
@@ -596,7 +601,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
                     const int i = (e * nblk + rank) * kThreads + threadIdx.x;
-                    if (i >= v.lead && i < n - v.w_eff && (level == 0 || (kb[e] >> (shift + 8)) == prefix)) {
+                    if (e < e_lim && i >= v.lead && i < n - v.w_eff && (level == 0 || (kb[e] >> (shift + 8)) == prefix)) {
                         const int dgt = (int)((kb[e] >> shift) & 255u);
                         atomicAdd(&sm.wcnt[warp][dgt], 1u);
                         add_u64_shared(&sm.wsum[warp][dgt], sq_fixed(kb[e], v.sbias));
@@ -692,6 +697,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
         __syncthreads();
 #pragma unroll
         for (int e = 0; e < E; ++e) {
+            if (e >= e_lim) continue;                                  // no run of this block there
             const int i = (e * nblk + rank) * kThreads + threadIdx.x;
             bool sure = false, tie = false;
             if (i < n) {
@@ -850,6 +856,11 @@ emit_kernel(refree_params p, const float *scores, const int32_t *seq_len, int64_
     __shared__ int s_pack;
     const int Hkv = p.num_kv_heads, U = p.num_seqs * Hkv;
     const int u = blockIdx.y, s = u / Hkv, g = u % Hkv;
+    // score ranking: a block beyond the end of its sequence has nothing to do (the grid is sized for the longest
+    // sequence a call can hold)
+    if (blockIdx.x > 0 && p.rank_mode != REFREE_RANK_POSITION && !p.force_full &&
+        (int64_t)blockIdx.x * kThreads >= max(seq_len[s], 0))
+        return;
     // offsets[u] = sum of lengths before u
     long long part = 0, off;
     for (int t = threadIdx.x; t < u; t += kThreads) part += lengths[t];
@@ -1029,9 +1040,10 @@ cudaError_t launch_select(const refree_params &p, const float *scores, const int
         // Score ranking per head: units short enough for a cluster to hold in registers go to the kernel that
         // reads the scores once; the general kernel takes the rest (all of them when none is short enough).
         if (p.rank_mode == REFREE_RANK_SCORE && !p.force_full && p.scope == REFREE_SCOPE_HEAD) {
-            int rb = nblk;                                   // blocks per unit: at least what the sizes call for
-            const int64_t want = std::min<int64_t>(total_tokens, (int64_t)kMaxCluster * kThreads * 16);
-            while (rb < kMaxCluster && (int64_t)rb * kThreads * 16 < want) rb *= 2;
+            // blocks per unit by the mean length, like the general kernel; elements per thread so that the longest
+            // sequence the call can hold fits if 16 allow it (longer units go to the general kernel)
+            const int rb = nblk;
+            const int64_t want = std::min<int64_t>(total_tokens, (int64_t)rb * kThreads * 16);
             int E = 4;
             while (E < 16 && (int64_t)rb * kThreads * E < want) E *= 2;
             cudaLaunchConfig_t rc = cfg;

@@ -24,10 +24,13 @@
 // exponential is taken.
 //
 // Persistent CTAs (one per SM) take contiguous ranges of (unit, tile) items; warp 16
-// issues TMA, warp 17 issues MMA, warps 0-15 are the epilogue.  Pass 1: four
-// accumulators of 128 columns, warps = (accumulator pair) x (64-column half).  Pass 2:
-// two accumulators of 256 columns, warps = (lane quarter) x (column chunk); the warps of
-// chunk 0 add the other chunks' column sums from shared memory one tile late.  Every
+// issues TMA, warp 17 issues MMA, warps 0-15 are the epilogue, warp 18 moves rows of
+// another layer, warps 19 and 20 finish the column pass.  Pass 1: four accumulators of
+// 128 columns, warps = (accumulator pair) x (64-column half).  Pass 2: two accumulators
+// of 256 columns, two groups of eight warps take the products in turn, a warp = (lane
+// quarter) x (half of the product's columns); the finishing warps add the warps' shares
+// of a tile, store the scores and the records of the stopping rule, tile by tile in
+// turn (one warp could not keep up with the sixteen: it paced the pass).  Every
 // wait is bounded: on a timeout the CTA records REFREE_DEV_TIMEOUT, stops issuing work,
 // and falls through to the common exit where tensor memory is released.
 #include <cuda.h>
@@ -43,7 +46,8 @@ namespace refree {
 namespace {
 
 constexpr int kEpiWarps = 16;
-constexpr int kThreadsTc = (kEpiWarps + 4) * 32;    // + TMA warp, MMA warp, copy warp, finishing warp
+constexpr int kFinishWarps = 1;                      // warps that finish the column pass, taking its tiles in turn
+constexpr int kThreadsTc = (kEpiWarps + 3 + kFinishWarps) * 32;    // + TMA warp, MMA warp, copy warp, finishing warps
 constexpr int kMaxCopySlots = 10;
 constexpr int kMaxCopyUnits = 1024;                 // units whose running budget sum fits the CTA's table
 constexpr int kD = 128;
@@ -219,18 +223,23 @@ struct ItemInfo {
     int32_t new_unit; // the item is the first of its unit in this CTA's pass
 };
 constexpr int kInfoRing = 16;   // the TMA thread runs at most ring stages + accumulators in flight ahead of the epilogue
+// Pass 2: tiles whose column sums wait for the finishing warp.  That warp is slower per tile than the sixteen
+// epilogue warps together while rows are being copied beside them, and catches up under the row pass that follows:
+// the ring is deep enough to let it fall behind instead of holding the epilogue back.
+constexpr int kStageSlots = 8;
 
 struct TcSmemTail {
     uint64_t k_full[4], k_empty[4], q_full, q_empty, epi_bar;
     uint64_t acc_full[4], acc_empty[4];       // pass 1: accumulator (pair * 2 + slot), 128 tensor-memory columns each
     uint64_t p2_full[2], p2_empty[2];         // pass 2: accumulators of 256 columns, one per group of eight warps
-    uint64_t chunk_ready[4];                  // pass 2: every share of a tile has been staged
-    uint64_t stage_free[4];                   // pass 2: the finishing warp has read the slot
+    uint64_t chunk_ready[kStageSlots];        // pass 2: every share of a tile has been staged
+    uint64_t stage_free[kStageSlots];         // pass 2: the finishing warp has read the slot
     uint64_t c_full[kMaxCopySlots];           // row copy: a piece has landed in its slot
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) ItemInfo info[kInfoRing];
-    alignas(16) float stage[4][4][kTile];     // pass 2: partial column sums (share = product * 2 + column half), four tiles deep
+    alignas(16) ItemInfo stage_info[kStageSlots];      // pass 2: the staged tile's record, copied beside its sums
+    alignas(16) float stage[kStageSlots][4][kTile];    // pass 2: partial column sums (share = product * 2 + column half)
     alignas(16) float lse[kMaxRowsTc];        // pass 2: log2-sum-exp of the unit's rows
 };
 
@@ -874,9 +883,12 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
                                     : col_job<true>(c_width >> 4, taddr, &tl.p2_empty[group], lane, scale, tl.lse,
                                                     cb * sh.ncol + c_begin, sh.R, w, pos_gap);
             // the slot's previous tile (four tiles ago) has been read by the finishing warp
-            const uint32_t slot = (uint32_t)item & 3u;
-            if (!(ok = mbar_wait(&tl.stage_free[slot], (((uint32_t)item >> 2) & 1u) ^ 1u, &tl.abort_flag))) break;
+            const uint32_t slot = (uint32_t)item % kStageSlots;
+            if (!(ok = mbar_wait(&tl.stage_free[slot], (((uint32_t)item / kStageSlots) & 1u) ^ 1u, &tl.abort_flag))) break;
             tl.stage[slot][cb * 2 + half][pos_in_tile] = part;
+            // the tile's record travels with its sums (the ring it came from may be reused before the tile is finished)
+            if (cb == 0 && half == 0 && lane_base == 0 && lane < 8)
+                reinterpret_cast<uint32_t *>(&tl.stage_info[slot])[lane] = reinterpret_cast<const uint32_t *>(inf)[lane];
             __syncwarp();
             if (lane == 0) mbar_arrive(&tl.chunk_ready[slot]);
         }
@@ -886,7 +898,7 @@ __device__ inline void epilogue_pass2(const TcArgs &a, TcSmemTail &tl, const Seq
 // Pass 2, the finishing warp: a'[i] = (sum of the warps' shares, in a fixed order) / (G * rows that see i)  (Eq. 2), the score
 // store, and per 32 positions the record the stopping rule reads.  `icount0` = items the roles have gone through
 // before this pass (their ring index).
-__device__ inline void finisher_pass2(const TcArgs &a, TcSmemTail &tl, int nitems, uint32_t icount0)
+__device__ inline void finisher_pass2(const TcArgs &a, TcSmemTail &tl, int nitems, uint32_t icount0, int which)
 {
     const int lane = threadIdx.x & 31;
     const int w = a.p.window;
@@ -920,15 +932,65 @@ __device__ inline void finisher_pass2(const TcArgs &a, TcSmemTail &tl, int nitem
         }
         run_tiles = 0;
     };
-    for (int t = 0; t < nitems; ++t) {
-        const uint32_t slot = (uint32_t)t & 3u;
-        if (!mbar_wait(&tl.chunk_ready[slot], ((uint32_t)t >> 2) & 1u, &tl.abort_flag)) return;
-        const ItemInfo *inf = &tl.info[(icount0 + (uint32_t)t) & (kInfoRing - 1)];
+    // tile t of the pass belongs to finishing warp t mod kFinishWarps; a warp counts and closes its own runs of a
+    // unit's tiles, and the unit is complete when the warps' counts add up to its tiles
+    for (int t = which; t < nitems; t += kFinishWarps) {
+        const uint32_t slot = (uint32_t)t % kStageSlots;
+        if (!mbar_wait(&tl.chunk_ready[slot], ((uint32_t)t / kStageSlots) & 1u, &tl.abort_flag)) return;
+        const ItemInfo *inf = &tl.stage_info[slot];
         const int n = inf->n, tile = inf->tile;
         const int inf_u = inf->u, inf_ntiles = inf->ntiles, inf_ib = inf->ib;     // the record may be reused after the slot is freed
         float *dst = a.scores + (int64_t)inf->g * a.total_tokens + inf->pack;
         GroupPartial *grp = a.groups ? a.groups + ((int64_t)inf->ib + tile) * 4 : nullptr;
         uint32_t tile_max = 0;
+        if ((reinterpret_cast<uintptr_t>(dst + (int64_t)tile * kTile) & 15) == 0) {
+            // A lane takes four consecutive positions: the shares come as 16-byte loads, the scores leave as one
+            // 16-byte store, and the 32 positions of a record are eight neighbouring lanes.  (Few instructions that
+            // go through the memory pipe: the sixteen epilogue warps keep it busy, and this warp paces the pass.)
+            const int p0 = 4 * lane, i0 = tile * kTile + p0;
+            float tot[4];
+            {
+                const float4 x = *reinterpret_cast<const float4 *>(&tl.stage[slot][0][p0]);
+                const float4 y = *reinterpret_cast<const float4 *>(&tl.stage[slot][1][p0]);
+                tot[0] = x.x + y.x; tot[1] = x.y + y.y; tot[2] = x.z + y.z; tot[3] = x.w + y.w;
+            }
+            if (two_products) {
+                const float4 x = *reinterpret_cast<const float4 *>(&tl.stage[slot][2][p0]);
+                const float4 y = *reinterpret_cast<const float4 *>(&tl.stage[slot][3][p0]);
+                tot[0] += x.x; tot[1] += x.y; tot[2] += x.z; tot[3] += x.w;
+                tot[0] += y.x; tot[1] += y.y; tot[2] += y.z; tot[3] += y.w;
+            }
+            float sc[4];
+            uint32_t bits[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = i0 + k;
+                const int cnt_i = max(1, min(min(w, n), n - i));
+                sc[k] = i < n ? tot[k] / ((float)cnt_i * g) : 0.f;
+                bits[k] = (i < n && isfinite(sc[k])) ? mag_bits(sc[k]) : 0u;
+                if (i < n && !isfinite(sc[k]) && a.dev_status) atomicOr(a.dev_status, REFREE_DEV_NONFINITE);
+            }
+            if (i0 + 3 < n) {
+                *reinterpret_cast<float4 *>(dst + i0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (i0 + k < n) dst[i0 + k] = sc[k];
+            }
+            if (grp) {
+                // 32 positions = lanes 8q .. 8q + 7: largest score, and the exact squares summed at a scale set by it
+                uint32_t mx = max(max(bits[0], bits[1]), max(bits[2], bits[3]));
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                const int shift = kGroupShift - 2 * max(1, (int)(mx >> 23));
+                unsigned long long sq = sq_fixed(bits[0], shift) + sq_fixed(bits[1], shift) + sq_fixed(bits[2], shift) +
+                                        sq_fixed(bits[3], shift);
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if ((lane & 7) == 0) { GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq; grp[lane >> 3] = gp; }
+                tile_max = __reduce_max_sync(0xffffffffu, mx);
+            }
+        } else {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const int pos = q * 32 + lane, i = tile * kTile + pos;
@@ -954,6 +1016,7 @@ __device__ inline void finisher_pass2(const TcArgs &a, TcSmemTail &tl, int nitem
                 for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
                 if (lane == 0) { GroupPartial gp; gp.max_bits = mx; gp.pad = 0u; gp.sum = sq; grp[q] = gp; }
             }
+        }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&tl.stage_free[slot]);
@@ -1124,7 +1187,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         mbar_init(&tl.q_empty, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(&tl.acc_full[b], 1); mbar_init(&tl.acc_empty[b], kEpiWarps / 2); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tl.p2_full[b], 1); mbar_init(&tl.p2_empty[b], kEpiWarps / 2); }
-        for (int b = 0; b < 4; ++b) {
+        for (int b = 0; b < kStageSlots; ++b) {
             mbar_init(&tl.chunk_ready[b], (kEpiWarps / 2) * a.sh.cblocks);      // eight warps stage a share per product
             mbar_init(&tl.stage_free[b], 1);
         }
@@ -1194,8 +1257,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mapq_a, const __grid_constan
         }
     } else if (warp == kEpiWarps + 2) {
         if (a.cj.nslots > 0) copy_loop(a, tl, sv, smem_c, coff);
-    } else if (warp == kEpiWarps + 3) {
-        if (P2) finisher_pass2(a, tl, nitems, MODE == 3 ? (uint32_t)nitems : 0u);
+    } else if (warp >= kEpiWarps + 3) {
+        if (P2) finisher_pass2(a, tl, nitems, MODE == 3 ? (uint32_t)nitems : 0u, warp - (kEpiWarps + 3));
     } else {
         if (lane == 0) {
             MmaState ms;

@@ -182,7 +182,7 @@ def algorithmic_bytes(cfg, seq_lens, lengths):
 # still has the hash it was captured on, and null afterwards.
 NCU_TRAFFIC = {
     # workload: (kernel source, first 16 hex digits of its sha256, bytes per launch)
-    "mistral7b_32k": ("paper_2502_16886_b200/csrc/score_tc.cu", "320db937c7063529", 262_295_296 + 97_656_320),
+    "mistral7b_32k": ("paper_2502_16886_b200/csrc/score_tc.cu", "848012eefce12c48", 262_343_936 + 92_841_216),
 }
 
 

@@ -761,8 +761,8 @@ def run_sweep(args):
     for window in (1, max(1, round(0.01 * n)), round(0.05 * n), round(0.10 * n)):
         cfg = dataclasses.replace(base, window=window)
         rows = cfg.group * window
-        if rows > 1024:
-            points += [{"window": window, "threshold": t, "status": "unsupported: G * window = %d rows > 1024" % rows}
+        if rows > 32768:
+            points += [{"window": window, "threshold": t, "status": "unsupported: G * window = %d rows > 32768" % rows}
                        for t in (0.001, 0.01, 0.1)]
             continue
         lays = [workloads.make_layer(cfg, l) for l in range(L)]

@@ -25,7 +25,10 @@
  *     reads device properties; make it outside any stream capture.
  *   - Limits, all reported as REFREE_ERR_UNSUPPORTED: num_seqs <= 1024;
  *     num_seqs * num_kv_heads <= 65535; (num_q_heads / num_kv_heads) * window
- *     <= 1024; head_dim 64 or 128; 16-byte aligned K/V base pointers and strides.
+ *     <= 32768 with at most 256 query heads per KV head (beyond 1024 query rows
+ *     per unit the window is scored in chunks of rows, K read once per chunk,
+ *     and the workspace holds one chunk's rows and scores more); head_dim 64 or
+ *     128; 16-byte aligned K/V base pointers and strides.
  *   - Element (s, g, i, :) of K lives at
  *       k + s*k_stride_seq + (seq_start[s] + i)*k_stride_tok + g*k_stride_head
  *     (strides in elements, head_dim contiguous); V likewise.  Rows

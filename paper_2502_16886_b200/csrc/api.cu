@@ -29,12 +29,23 @@ int sm_count()
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Window rows scored at once: the whole window when a scoring path takes it, else a chunk that one does
+// (512 query rows on the tensor-core path, 1024 on the generic one).
+static int chunk_window(const refree_params &p)
+{
+    const int G = p.num_q_heads / p.num_kv_heads;
+    if ((int64_t)G * p.window <= kMaxRows) return p.window;
+    const int cap = (p.dtype == REFREE_DTYPE_BF16 && p.head_dim == 128) ? 512 : kMaxRows;
+    return std::max(1, cap / G);
+}
+
 Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
 {
     Workspace w;
     const int64_t U = (int64_t)p.num_seqs * p.num_kv_heads;
     const int64_t G = p.num_q_heads / p.num_kv_heads;
-    const int64_t rows = G * p.window;
+    const int wc = chunk_window(p);
+    const int64_t rows = G * wc;
     const int64_t tiles = total_tokens / kTile + p.num_seqs;
     size_t off = 0;
     // partials: per (tile, head, row) for the generic path, per (CTA + unit, column half, padded row) for the tensor-core path
@@ -49,6 +60,14 @@ Workspace workspace_layout(const refree_params &p, int64_t total_tokens)
     w.cut_off = off;    w.cut_bytes = align256((size_t)U * sizeof(Cut));                                   off += w.cut_bytes;
     w.scores_off = off; w.scores_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)); off += w.scores_bytes;
     w.kept_off = off;   w.kept_bytes = align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(int32_t)); off += w.kept_bytes;
+    w.chk_off = off;    w.chk_bytes = 0;
+    if (wc < p.window) {
+        const size_t esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+        w.chk_bytes = align256((size_t)p.num_seqs * p.num_q_heads * wc * p.head_dim * esz) +
+                      align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)) +
+                      align256((size_t)p.num_seqs * sizeof(int32_t));
+    }
+    off += w.chk_bytes;
     w.total = off;
     return w;
 }
@@ -67,7 +86,10 @@ static refree_status check_params(const refree_params *p, int64_t total_tokens)
     if (p->head_dim != 64 && p->head_dim != 128) return REFREE_ERR_UNSUPPORTED;
     if (p->num_seqs > kMaxSeqs) return REFREE_ERR_UNSUPPORTED;
     if ((int64_t)p->num_seqs * p->num_kv_heads > 65535) return REFREE_ERR_UNSUPPORTED;
-    if ((int64_t)(p->num_q_heads / p->num_kv_heads) * p->window > kMaxRows) return REFREE_ERR_UNSUPPORTED;
+    if ((int64_t)(p->num_q_heads / p->num_kv_heads) * p->window > kMaxRows &&
+        ((int64_t)(p->num_q_heads / p->num_kv_heads) * p->window > kMaxRowsChunked ||
+         p->num_q_heads / p->num_kv_heads > kMaxGroupChunked))
+        return REFREE_ERR_UNSUPPORTED;
     return REFREE_OK;
 }
 
@@ -96,11 +118,78 @@ static bool use_tc(const refree_params &p, const void *q_win)
     return score_tc_supported(p) && !(reinterpret_cast<uintptr_t>(q_win) & 15);
 }
 
+namespace {
+// Lengths of the sequences as a chunk of window rows sees them: cut after the chunk's last row.
+__global__ void chunk_lens_kernel(const int32_t *seq_len, int32_t *len_c, int num_seqs, int rows_after)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < num_seqs) len_c[s] = max(0, max(seq_len[s], 0) - rows_after);
+}
+
+// scores += chunk scores * (chunk rows that see the position), i.e. the chunk's column sums over G; the last
+// chunk divides by the rows of the whole window that see the position (Eq. 2).
+__global__ void chunk_accumulate_kernel(refree_params p, const int32_t *seq_len, const int32_t *len_c, const float *sc,
+                                        float *scores, int64_t total_tokens, int wc, int last)
+{
+    __shared__ int s_pack, s_pack_c;
+    const int Hkv = p.num_kv_heads, s = blockIdx.y / Hkv, g = blockIdx.y % Hkv;
+    if (threadIdx.x == 0) {
+        int a = 0, b = 0;
+        for (int t = 0; t < s; ++t) { a += max(seq_len[t], 0); b += len_c[t]; }
+        s_pack = a;
+        s_pack_c = b;
+    }
+    __syncthreads();
+    const int n = max(seq_len[s], 0), nc = len_c[s];
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        float acc = scores[(int64_t)g * total_tokens + s_pack + i];
+        if (i < nc) {
+            const int cnt_c = max(1, min(min(wc, nc), nc - i));
+            acc += sc[(int64_t)g * total_tokens + s_pack_c + i] * (float)cnt_c;
+        }
+        if (last) acc /= (float)max(1, min(min(p.window, n), n - i));
+        scores[(int64_t)g * total_tokens + s_pack + i] = acc;
+    }
+}
+}  // namespace
+
 static cudaError_t run_score(const refree_params &p, const void *q_win, const void *k,
                              const int32_t *seq_start, const int32_t *seq_len, int64_t total_tokens,
                              float *scores, char *ws, const Workspace &lay, int32_t *dev_status,
                              cudaStream_t st, GroupPartial *groups = nullptr)
 {
+    const int wc = chunk_window(p);
+    if (wc < p.window) {
+        // Window too long for one pass: chunks of window rows from the last backwards, each scored as a window of
+        // its own over the sequences cut at its last row (K is read again per chunk), then weighted back to column
+        // sums and added up.  The chunks' scores are exact column sums up to one rounding each.
+        const size_t esz = p.dtype == REFREE_DTYPE_F32 ? 4 : 2;
+        const size_t row_bytes = (size_t)p.head_dim * esz;
+        char *qc = ws + lay.chk_off;
+        float *sc = reinterpret_cast<float *>(qc + align256((size_t)p.num_seqs * p.num_q_heads * wc * row_bytes));
+        int32_t *len_c = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(sc) +
+                                                    align256((size_t)(p.num_kv_heads * total_tokens) * sizeof(float)));
+        cudaError_t e = cudaMemsetAsync(scores, 0, (size_t)(p.num_kv_heads * total_tokens) * sizeof(float), st);
+        if (e != cudaSuccess) return e;
+        const int gx = (int)std::min<int64_t>(1024, (total_tokens + 255) / 256);
+        for (int t1 = p.window; t1 > 0; t1 -= wc) {
+            const int t0 = std::max(0, t1 - wc), wcur = t1 - t0;
+            refree_params pc = p;
+            pc.window = wcur;
+            e = cudaMemcpy2DAsync(qc, (size_t)wcur * row_bytes, (const char *)q_win + (size_t)t0 * row_bytes,
+                                  (size_t)p.window * row_bytes, (size_t)wcur * row_bytes,
+                                  (size_t)p.num_seqs * p.num_q_heads, cudaMemcpyDeviceToDevice, st);
+            if (e != cudaSuccess) return e;
+            chunk_lens_kernel<<<(p.num_seqs + 255) / 256, 256, 0, st>>>(seq_len, len_c, p.num_seqs, p.window - t1);
+            count_launches(1);
+            e = run_score(pc, qc, k, seq_start, len_c, total_tokens, sc, ws, lay, dev_status, st, nullptr);
+            if (e != cudaSuccess) return e;
+            chunk_accumulate_kernel<<<dim3(gx, p.num_seqs * p.num_kv_heads), 256, 0, st>>>(p, seq_len, len_c, sc, scores,
+                                                                                         total_tokens, wcur, t0 == 0);
+            count_launches(1);
+        }
+        return cudaGetLastError();
+    }
     if (use_tc(p, q_win))
         return launch_score_tc(p, q_win, k, seq_start, seq_len, total_tokens, scores, ws, lay, dev_status, st, groups);
     if (score_w1_supported(p))

@@ -12,6 +12,10 @@ namespace refree {
 constexpr int kMaxSeqs = 1024;   // sequences per call (prefix tables live in shared memory)
 constexpr int kTile = 128;       // positions per scoring tile
 constexpr int kMaxRows = 1024;   // G * window handled by the generic scoring path
+// Longer windows (Section 4.4 studies windows of up to a tenth of the sequence) are scored in chunks of query rows
+// that the scoring paths take, each chunk a window of its own over a sequence cut at its last row.
+constexpr int kMaxRowsChunked = 32768;
+constexpr int kMaxGroupChunked = 256;   // query heads per KV head when the window is chunked
 
 // Bounded spin: polls before a wait gives up and reports REFREE_DEV_TIMEOUT.
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -31,6 +35,7 @@ struct Workspace {
     size_t cut_off, cut_bytes;         // per unit selection result (struct Cut)
     size_t scores_off, scores_bytes;   // scratch scores when the caller passes none
     size_t kept_off, kept_bytes;       // scratch kept_idx when the caller passes none
+    size_t chk_off, chk_bytes;         // chunked windows: one chunk's query rows, its scores, its sequence lengths
     size_t total;
 };
 

@@ -144,3 +144,24 @@ def test_position_ranking_beyond_the_length_the_record_fed_rule_takes():
     cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=2, num_kv_heads=1, window=16, heavy_count=300)
     lay = workloads.make_layer(cfg, 0, seq_lens=[140_000, 700])
     parity.run_fused_and_check(cfg, lay)
+
+
+@pytest.mark.parametrize("kind", ["tensor_core_chunks", "generic_chunks"])
+@pytest.mark.parametrize("rank_mode", [binding.RANK_POSITION, binding.RANK_SCORE])
+def test_windows_longer_than_one_scoring_pass_are_scored_in_chunks(kind, rank_mode):
+    # Section 4.4 studies windows of up to a tenth of the sequence: G * w beyond 1024 query rows is scored in
+    # chunks of window rows (512 rows on the tensor-core path, 1024 on the generic one), the last chunk ragged,
+    # with one sequence shorter than the window and one shorter than a chunk
+    if kind == "tensor_core_chunks":
+        cfg = cfg_like(dtype="bf16", head_dim=128, num_q_heads=8, num_kv_heads=2, window=300, heavy_count=60)
+    else:
+        cfg = cfg_like(num_q_heads=4, num_kv_heads=2, window=1100, heavy_count=60)
+    lay = workloads.make_layer(cfg, 0, seq_lens=[3000, 200, 0, 90])
+    parity.run_fused_and_check(cfg, lay, rank_mode=rank_mode)
+
+
+def test_rows_beyond_what_chunks_cover_are_refused():
+    p = binding.Params(num_seqs=1, num_q_heads=4, num_kv_heads=1, head_dim=64, window=10_000, dtype=binding.DTYPE_F32,
+                       kv_tokens=16, k_strides=(0, 64, 16 * 64), v_strides=(0, 64, 16 * 64))
+    with pytest.raises(binding.RefreeError):
+        binding.refree_workspace_size(p, 16)

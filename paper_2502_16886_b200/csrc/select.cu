@@ -223,6 +223,7 @@ struct SelectSmem {
     unsigned int dabv_c[8], ddig[8];
     uint32_t y_mx;                    // fixed point, exchanged once: a block's largest key and its sum of squares
     float y_acc;                      // at that key's scale
+    uint32_t z_key;                   // the crossing key, told by the block that holds it when one position has it
     unsigned int wcnt[kWarps][257];   // per-warp private histograms (padded: one bank per warp for a digit)
     u64 wsum[kWarps][257];
     int pack;
@@ -482,6 +483,7 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
         int a = 0;
         for (int t = 0; t < s; ++t) a += max(seq_len[t], 0);
         sm.pack = a;
+        sm.z_key = 0u;
     }
     __syncthreads();
     const int n = max(seq_len[s], 0);
@@ -595,7 +597,8 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
             };
             clear_hist();
             __syncthreads();
-            for (int level = 0; level < 4 && any; ++level) {
+            bool spelled = false;             // the crossing key is known in full before the last level
+            for (int level = 0; level < 4 && any && !spelled; ++level) {
                 const int shift = 24 - 8 * level;
                 const int hb = level & 1;
 #pragma unroll
@@ -668,6 +671,27 @@ select_score_resident_kernel(refree_params p, const float *scores, const int32_t
                     above_sum += sm.dabv_s[cw];
                     above_cnt += sm.dabv_c[cw];
                     digit_cnt = (int)sm.ddig[cw];
+                    if (digit_cnt == 1 && level < 3) {
+                        // One position has the crossing digits: the remaining levels would only spell out its key.
+                        // The thread that holds it says it; every block reads it after one barrier.
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            const int i = (e * nblk + rank) * kThreads + threadIdx.x;
+                            if (e < e_lim && i >= v.lead && i < n - v.w_eff && (kb[e] >> shift) == prefix) sm.z_key = kb[e];
+                        }
+                        uint32_t key = 0u;
+                        if (nblk > 1) {
+                            cl.sync();
+#pragma unroll
+                            for (int b = 0; b < kMaxCluster; ++b)
+                                if (b < nblk) key = max(key, *cl.map_shared_rank(&sm.z_key, b));
+                        } else {
+                            __syncthreads();
+                            key = sm.z_key;
+                        }
+                        prefix = key;
+                        spelled = true;
+                    }
                 }
             }
             if (any) {

@@ -255,7 +255,8 @@ def test_pipelined_host_run_of_layers_matches_the_per_layer_call(rank_mode, pinn
 
 
 @pytest.mark.parametrize("rank_mode,window,dtype", [(binding.RANK_POSITION, 16, "bf16"), (binding.RANK_SCORE, 16, "bf16"),
-                                                    (binding.RANK_POSITION, 1, "bf16"), (binding.RANK_POSITION, 8, "fp32")])
+                                                    (binding.RANK_POSITION, 1, "bf16"), (binding.RANK_POSITION, 8, "fp32"),
+                                                    (binding.RANK_POSITION, 300, "bf16")])    # 1200 query rows: scored in chunks
 def test_pipelined_device_run_of_layers_matches_the_per_layer_call(rank_mode, window, dtype):
     """refree_compress_layers (scoring of layer l + 1 over the compaction of layer l, two internal
     streams, two workspace halves) against one refree_compress_layer call per layer: five layers, so
